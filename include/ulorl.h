@@ -1,0 +1,153 @@
+/*
+ * ulorl.h -- C ABI of the fused UloRL token-loss library (CUDA, sm_100a).
+ *
+ * One call pair computes, for T packed response tokens, the per-token part of the UloRL
+ * policy update: LM-head logits z = kappa * hidden W^T, log-softmax and entropy per
+ * token (the policy of Eq. 6 and the vocabulary sum of Eq. 10's H-bar), the segment-aware
+ * or pseudo-on-policy importance ratio (Eq. 8, Section 3.1.2), the well-mastered-positive-
+ * token mask (Eq. 9) under the entropy gate of Eq. 10, the clipped token-normalised
+ * surrogate (Eq. 10 with the bounds of Eq. 7), and its gradients to hidden and W.
+ * The T x V logits are never written to global memory.
+ *
+ * Conventions
+ *  - Every pointer except `params` is DEVICE memory owned by the caller, row-major and
+ *    contiguous.  The library allocates nothing, frees nothing and keeps no state
+ *    between calls.
+ *  - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*) and never
+ *    synchronise.  `loss` and `stats` stay on the device.
+ *  - The return value is the host-side validation / launch status.  Device-side problems
+ *    (a target outside [0, V), a bounded wait that ran out) are recorded in a status word
+ *    inside the workspace and read back by ulorl_check_status(); offending rows are
+ *    clamped, never read out of bounds.
+ *  - Tokens are response tokens only; there is no ignore-index.
+ *  - hidden, W and d_hidden have the element type `dtype`.  H must be a multiple of 8.
+ */
+#ifndef ULORL_H_
+#define ULORL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  ULORL_OK = 0,
+  ULORL_ERR_INVALID_ARG = -1,   /* NULL pointer, negative size, inconsistent offsets    */
+  ULORL_ERR_UNSUPPORTED = -2,   /* shape / dtype / alignment the kernels do not cover   */
+  ULORL_ERR_WORKSPACE = -3,     /* workspace smaller than ulorl_workspace_bytes()       */
+  ULORL_ERR_CUDA = -4,          /* a CUDA runtime or driver call failed                 */
+  ULORL_ERR_DEVICE_TIMEOUT = -5,/* a bounded device-side wait ran out                   */
+  ULORL_ERR_BAD_TARGET = -6     /* some target id was outside [0, V) (row was clamped)  */
+} ulorl_status_t;
+
+typedef enum { ULORL_F32 = 0, ULORL_BF16 = 1 } ulorl_dtype_t;
+typedef enum { ULORL_IS_SAIS = 0, ULORL_IS_POIS = 1 } ulorl_is_mode_t;            /* Eq. 8 | Section 3.1.2 */
+typedef enum { ULORL_MPT_OFF = 0, ULORL_MPT_ALWAYS = 1, ULORL_MPT_DYNAMIC = 2 } ulorl_mpt_mode_t; /* Section 3.2 */
+typedef enum { ULORL_ENT_PER_SEQ = 0, ULORL_ENT_BATCH = 1, ULORL_ENT_SUPPLIED = 2 } ulorl_ent_scope_t;
+typedef enum { ULORL_PATH_AUTO = 0, ULORL_PATH_SIMT = 1, ULORL_PATH_TENSOR = 2 } ulorl_kernel_path_t;
+
+/* bits of flags[t] */
+#define ULORL_FLAG_MASKED    1u  /* MPT and gate open: excluded from the objective (Eq. 10)   */
+#define ULORL_FLAG_CLIP_HIGH 2u  /* A > 0 and ratio > 1 + eps_high: gradient clipped           */
+#define ULORL_FLAG_CLIP_LOW  4u  /* A < 0 and ratio < 1 - eps_low : gradient clipped           */
+#define ULORL_FLAG_MPT       8u  /* well-mastered positive token (Eq. 9), whatever the gate    */
+
+#define ULORL_N_STALENESS 16
+
+typedef struct {
+  int32_t T, H, V, num_seqs;   /* packed tokens, hidden size, vocabulary, sequences (seq_offsets[num_seqs] == T) */
+  int32_t dtype;               /* ulorl_dtype_t of hidden, W, d_hidden                                           */
+  int32_t is_mode;             /* ulorl_is_mode_t                                                                */
+  int32_t mpt_mode;            /* ulorl_mpt_mode_t                                                               */
+  int32_t ent_scope;           /* ulorl_ent_scope_t: which entropy the gate H-bar < sigma is taken on            */
+  int32_t adv_per_token;       /* 0: advantages[num_seqs]; 1: advantages[T]                                      */
+  float clip_eps_low;          /* Eq. 7 bounds; the paper gives no value, workloads use 0.2 / 0.2                */
+  float clip_eps_high;
+  float mpt_tau;               /* probability threshold of Eq. 9 (0.99 in Section 4.1)                           */
+  float entropy_target;        /* sigma of Eq. 10 (0.2 in Section 4.1)                                           */
+  float inv_temperature;       /* kappa multiplying the logits; 1 unless the caller trains at a temperature      */
+  int64_t norm_tokens;         /* N of Eq. 10; 0 means T (a micro-batch passes the global token count)           */
+  int32_t current_version;     /* id of the latest policy; staleness = current_version - segment_version[t]      */
+  int32_t dw_accumulate;       /* bwd: 0 overwrite d_W, 1 add into it (micro-batching)                           */
+  int32_t kernel_path;         /* ulorl_kernel_path_t; AUTO = tensor-core path for bf16, SIMT path for f32       */
+  int32_t bwd_panel_tokens;    /* bwd: tokens per staging panel; 0 = library default                             */
+} ulorl_params_t;
+
+typedef struct {
+  float loss;                  /* -(1/N) sum_t (1 - msk_t) s_t                                                    */
+  float mean_entropy;          /* token mean of the per-token entropy over the call                               */
+  int32_t n_tokens, n_active, n_mpt, n_masked, n_clip_high, n_clip_low;
+  int32_t stale_tokens[ULORL_N_STALENESS];     /* tokens per staleness bucket (last bucket = that or more)        */
+  int32_t stale_clipped[ULORL_N_STALENESS];    /* of which clipped                                                */
+  float stale_mean_abs_logratio[ULORL_N_STALENESS];
+  int32_t device_status;       /* copy of the workspace status word at the end of the forward call                */
+  int32_t reserved[3];
+} ulorl_stats_t;
+
+/* Bytes of workspace both calls need for these params (pure host function; 0 on invalid params). */
+size_t ulorl_workspace_bytes(const ulorl_params_t* params);
+
+/*
+ * Forward (Eq. 6, 8, 9, 10).  Inputs:
+ *   hidden [T,H], W [V,H]  element type params->dtype
+ *   targets [T] int32      generated token ids y_t
+ *   old_logp [T] f32       log-prob recorded at rollout by the policy that generated the token's
+ *                          segment (Eq. 8); may be NULL in POIS mode
+ *   segment_version [T]    id of that policy (statistics only); may be NULL
+ *   advantages             f32, [num_seqs] or [T] (adv_per_token)
+ *   seq_offsets [S+1]      int32, non-decreasing, seq_offsets[0] = 0, seq_offsets[S] = T
+ *   entropy_supplied [S]   f32 gate values, read only when ent_scope = SUPPLIED
+ * Outputs (all f32 unless noted; any of logp/entropy/lse/grad_coef/flags/seq_entropy must be non-NULL):
+ *   logp[T], entropy[T], lse[T], grad_coef[T] (= d loss / d logp_t, saved for bwd),
+ *   flags[T] uint8, seq_entropy[S] (H-bar_i), loss[1], stats (ulorl_stats_t, may be NULL).
+ */
+int ulorl_token_loss_fwd(const ulorl_params_t* params,
+                         const void* hidden, const void* W, const int32_t* targets,
+                         const float* old_logp, const int32_t* segment_version,
+                         const float* advantages, const int32_t* seq_offsets,
+                         const float* entropy_supplied,
+                         float* logp, float* entropy, float* lse, float* grad_coef,
+                         uint8_t* flags, float* seq_entropy, float* loss, void* stats,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * The elementwise stage alone (Eq. 8, 9, 10 given per-token log-prob and entropy): per-sequence
+ * mean entropy, ratio, mask, clipped surrogate, loss, d loss / d logp.  Same arguments as the
+ * forward call with logp[T] and entropy[T] as INPUTS.
+ */
+int ulorl_token_loss_decide(const ulorl_params_t* params,
+                            const float* logp, const float* entropy,
+                            const float* old_logp, const int32_t* segment_version,
+                            const float* advantages, const int32_t* seq_offsets,
+                            const float* entropy_supplied,
+                            float* grad_coef, uint8_t* flags, float* seq_entropy, float* loss,
+                            void* stats, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Backward (chain rule through Eq. 6): with dz[t,v] = kappa * grad_loss * grad_coef[t] *
+ * (1[v = y_t] - exp(z[t,v] - lse[t])), writes d_hidden[T,H] (params->dtype) and d_W[V,H] (f32;
+ * added into when params->dw_accumulate).  grad_loss is a device scalar or NULL (= 1).
+ * Logits are recomputed tile by tile; nothing of size T x V is kept beyond one token panel
+ * of dz in the workspace.
+ */
+int ulorl_token_loss_bwd(const ulorl_params_t* params,
+                         const void* hidden, const void* W, const int32_t* targets,
+                         const float* lse, const float* grad_coef, const float* grad_loss,
+                         void* d_hidden, float* d_W,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Synchronises the stream, reads the workspace status word and returns it (ULORL_OK, or
+ * ULORL_ERR_DEVICE_TIMEOUT / ULORL_ERR_BAD_TARGET / ULORL_ERR_CUDA). */
+int ulorl_check_status(void* workspace, void* cuda_stream);
+
+const char* ulorl_status_string(int status);
+
+/* Number of kernel launches issued by this library since it was loaded (host counter). */
+int64_t ulorl_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ULORL_H_ */

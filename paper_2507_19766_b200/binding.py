@@ -1,0 +1,264 @@
+"""ctypes binding of libulorl.so: argument marshalling only.
+
+Every step of the token-loss path runs inside the CUDA library; this module turns torch
+tensors into device pointers, fills the parameter struct and checks return codes.  There is
+no CPU fallback: if the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libulorl.so")
+
+OK = 0
+F32, BF16 = 0, 1
+IS_SAIS, IS_POIS = 0, 1
+MPT_OFF, MPT_ALWAYS, MPT_DYNAMIC = 0, 1, 2
+ENT_PER_SEQ, ENT_BATCH, ENT_SUPPLIED = 0, 1, 2
+PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
+FLAG_MASKED, FLAG_CLIP_HIGH, FLAG_CLIP_LOW, FLAG_MPT = 1, 2, 4, 8
+N_STALENESS = 16
+
+_IS = {"sais": IS_SAIS, "pois": IS_POIS}
+_MPT = {"off": MPT_OFF, "always": MPT_ALWAYS, "dynamic": MPT_DYNAMIC}
+_ENT = {"per_seq": ENT_PER_SEQ, "batch": ENT_BATCH, "supplied": ENT_SUPPLIED}
+_PATH = {"auto": PATH_AUTO, "simt": PATH_SIMT, "tensor": PATH_TENSOR}
+
+
+class UlorlError(RuntimeError):
+    pass
+
+
+class CParams(ctypes.Structure):
+    _fields_ = [
+        ("T", ctypes.c_int32), ("H", ctypes.c_int32), ("V", ctypes.c_int32), ("num_seqs", ctypes.c_int32),
+        ("dtype", ctypes.c_int32), ("is_mode", ctypes.c_int32), ("mpt_mode", ctypes.c_int32),
+        ("ent_scope", ctypes.c_int32), ("adv_per_token", ctypes.c_int32),
+        ("clip_eps_low", ctypes.c_float), ("clip_eps_high", ctypes.c_float), ("mpt_tau", ctypes.c_float),
+        ("entropy_target", ctypes.c_float), ("inv_temperature", ctypes.c_float),
+        ("norm_tokens", ctypes.c_int64), ("current_version", ctypes.c_int32),
+        ("dw_accumulate", ctypes.c_int32), ("kernel_path", ctypes.c_int32), ("bwd_panel_tokens", ctypes.c_int32),
+    ]
+
+
+class CStats(ctypes.Structure):
+    _fields_ = [
+        ("loss", ctypes.c_float), ("mean_entropy", ctypes.c_float),
+        ("n_tokens", ctypes.c_int32), ("n_active", ctypes.c_int32), ("n_mpt", ctypes.c_int32),
+        ("n_masked", ctypes.c_int32), ("n_clip_high", ctypes.c_int32), ("n_clip_low", ctypes.c_int32),
+        ("stale_tokens", ctypes.c_int32 * N_STALENESS), ("stale_clipped", ctypes.c_int32 * N_STALENESS),
+        ("stale_mean_abs_logratio", ctypes.c_float * N_STALENESS),
+        ("device_status", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3),
+    ]
+
+
+EXPORTS = ("ulorl_workspace_bytes", "ulorl_token_loss_fwd", "ulorl_token_loss_decide", "ulorl_token_loss_bwd",
+           "ulorl_check_status", "ulorl_status_string", "ulorl_launch_count")
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libulorl.so (built in-tree by paper_2507_19766_b200/build.py).  Raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise UlorlError(f"{LIB_PATH} is missing: build it with `python -m paper_2507_19766_b200.build` "
+                         "(there is no CPU fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, cp = ctypes.c_void_p, ctypes.POINTER(CParams)
+    lib.ulorl_workspace_bytes.restype = ctypes.c_size_t
+    lib.ulorl_workspace_bytes.argtypes = [cp]
+    lib.ulorl_token_loss_fwd.restype = ctypes.c_int
+    lib.ulorl_token_loss_fwd.argtypes = [cp] + [vp] * 16 + [vp, ctypes.c_size_t, vp]
+    lib.ulorl_token_loss_decide.restype = ctypes.c_int
+    lib.ulorl_token_loss_decide.argtypes = [cp] + [vp] * 12 + [vp, ctypes.c_size_t, vp]
+    lib.ulorl_token_loss_bwd.restype = ctypes.c_int
+    lib.ulorl_token_loss_bwd.argtypes = [cp] + [vp] * 8 + [vp, ctypes.c_size_t, vp]
+    lib.ulorl_check_status.restype = ctypes.c_int
+    lib.ulorl_check_status.argtypes = [vp, vp]
+    lib.ulorl_status_string.restype = ctypes.c_char_p
+    lib.ulorl_status_string.argtypes = [ctypes.c_int]
+    lib.ulorl_launch_count.restype = ctypes.c_int64
+    lib.ulorl_launch_count.argtypes = []
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load_library().ulorl_status_string(code).decode()
+
+
+def _check(code: int, what: str):
+    if code != OK:
+        raise UlorlError(f"{what} failed: {status_string(code)} ({code})")
+
+
+@dataclass
+class Params:
+    """Mirror of ulorl_params_t with the paper's names (Eq. 7-10, Section 4.1)."""
+    T: int
+    H: int
+    V: int
+    num_seqs: int
+    dtype: str = "bf16"
+    is_mode: str = "sais"
+    mpt_mode: str = "dynamic"
+    ent_scope: str = "per_seq"
+    adv_per_token: bool = False
+    clip_eps_low: float = 0.2
+    clip_eps_high: float = 0.2
+    mpt_tau: float = 0.99
+    entropy_target: float = 0.2
+    inv_temperature: float = 1.0
+    norm_tokens: int = 0
+    current_version: int = 0
+    dw_accumulate: bool = False
+    kernel_path: str = "auto"
+    bwd_panel_tokens: int = 0
+
+    def to_c(self) -> CParams:
+        return CParams(self.T, self.H, self.V, self.num_seqs, BF16 if self.dtype == "bf16" else F32,
+                       _IS[self.is_mode], _MPT[self.mpt_mode], _ENT[self.ent_scope], int(self.adv_per_token),
+                       self.clip_eps_low, self.clip_eps_high, self.mpt_tau, self.entropy_target,
+                       self.inv_temperature, self.norm_tokens, self.current_version, int(self.dw_accumulate),
+                       _PATH[self.kernel_path], self.bwd_panel_tokens)
+
+
+def workspace_bytes(p: Params) -> int:
+    n = load_library().ulorl_workspace_bytes(ctypes.byref(p.to_c()))
+    if n == 0:
+        raise UlorlError("ulorl_workspace_bytes: invalid parameters")
+    return int(n)
+
+
+def launch_count() -> int:
+    return int(load_library().ulorl_launch_count())
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise UlorlError("tensors must be contiguous CUDA tensors")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _want(t: torch.Tensor, dtype, n: int, name: str):
+    if t.dtype != dtype or t.numel() != n:
+        raise UlorlError(f"{name}: expected {n} elements of {dtype}, got {t.numel()} of {t.dtype}")
+
+
+@dataclass
+class FwdOut:
+    logp: torch.Tensor
+    entropy: torch.Tensor
+    lse: torch.Tensor
+    grad_coef: torch.Tensor
+    flags: torch.Tensor
+    seq_entropy: torch.Tensor
+    loss: torch.Tensor
+    stats: torch.Tensor      # raw bytes of ulorl_stats_t on the device
+
+    def stats_host(self) -> dict:
+        return decode_stats(self.stats)
+
+
+def decode_stats(stats: torch.Tensor) -> dict:
+    raw = bytes(stats.cpu().numpy().tobytes())
+    s = CStats.from_buffer_copy(raw)
+    return dict(loss=s.loss, mean_entropy=s.mean_entropy, n_tokens=s.n_tokens, n_active=s.n_active, n_mpt=s.n_mpt,
+                n_masked=s.n_masked, n_clip_high=s.n_clip_high, n_clip_low=s.n_clip_low,
+                stale_tokens=list(s.stale_tokens), stale_clipped=list(s.stale_clipped),
+                stale_mean_abs_logratio=list(s.stale_mean_abs_logratio), device_status=s.device_status)
+
+
+def alloc_workspace(p: Params, device) -> torch.Tensor:
+    return torch.empty(workspace_bytes(p), dtype=torch.uint8, device=device)
+
+
+def alloc_fwd_outputs(p: Params, device) -> FwdOut:
+    f = dict(dtype=torch.float32, device=device)
+    return FwdOut(logp=torch.empty(p.T, **f), entropy=torch.empty(p.T, **f), lse=torch.empty(p.T, **f),
+                  grad_coef=torch.empty(p.T, **f), flags=torch.empty(p.T, dtype=torch.uint8, device=device),
+                  seq_entropy=torch.empty(max(p.num_seqs, 1), **f), loss=torch.empty(1, **f),
+                  stats=torch.empty(ctypes.sizeof(CStats), dtype=torch.uint8, device=device))
+
+
+def token_loss_fwd(p: Params, hidden, W, targets, old_logp, segment_version, advantages, seq_offsets,
+                   entropy_supplied=None, out: Optional[FwdOut] = None, workspace: Optional[torch.Tensor] = None) -> FwdOut:
+    """ulorl_token_loss_fwd on the current CUDA stream."""
+    lib = load_library()
+    dev = hidden.device
+    tdt = torch.bfloat16 if p.dtype == "bf16" else torch.float32
+    _want(hidden, tdt, p.T * p.H, "hidden")
+    _want(W, tdt, p.V * p.H, "W")
+    _want(targets, torch.int32, p.T, "targets")
+    _want(seq_offsets, torch.int32, p.num_seqs + 1, "seq_offsets")
+    _want(advantages, torch.float32, p.T if p.adv_per_token else p.num_seqs, "advantages")
+    if old_logp is not None:
+        _want(old_logp, torch.float32, p.T, "old_logp")
+    if segment_version is not None:
+        _want(segment_version, torch.int32, p.T, "segment_version")
+    out = out or alloc_fwd_outputs(p, dev)
+    workspace = workspace if workspace is not None else alloc_workspace(p, dev)
+    code = lib.ulorl_token_loss_fwd(
+        ctypes.byref(p.to_c()), _ptr(hidden), _ptr(W), _ptr(targets), _ptr(old_logp), _ptr(segment_version),
+        _ptr(advantages), _ptr(seq_offsets), _ptr(entropy_supplied), _ptr(out.logp), _ptr(out.entropy), _ptr(out.lse),
+        _ptr(out.grad_coef), _ptr(out.flags), _ptr(out.seq_entropy), _ptr(out.loss), _ptr(out.stats),
+        _ptr(workspace), workspace.numel(), _stream())
+    _check(code, "ulorl_token_loss_fwd")
+    return out
+
+
+def token_loss_decide(p: Params, logp, entropy, old_logp, segment_version, advantages, seq_offsets,
+                      entropy_supplied=None, out: Optional[FwdOut] = None,
+                      workspace: Optional[torch.Tensor] = None) -> FwdOut:
+    """ulorl_token_loss_decide: the elementwise stage on given per-token log-probs and entropies."""
+    lib = load_library()
+    dev = logp.device
+    _want(logp, torch.float32, p.T, "logp")
+    _want(entropy, torch.float32, p.T, "entropy")
+    out = out or alloc_fwd_outputs(p, dev)
+    out.logp, out.entropy = logp, entropy
+    workspace = workspace if workspace is not None else alloc_workspace(p, dev)
+    code = lib.ulorl_token_loss_decide(
+        ctypes.byref(p.to_c()), _ptr(logp), _ptr(entropy), _ptr(old_logp), _ptr(segment_version), _ptr(advantages),
+        _ptr(seq_offsets), _ptr(entropy_supplied), _ptr(out.grad_coef), _ptr(out.flags), _ptr(out.seq_entropy),
+        _ptr(out.loss), _ptr(out.stats), _ptr(workspace), workspace.numel(), _stream())
+    _check(code, "ulorl_token_loss_decide")
+    return out
+
+
+def token_loss_bwd(p: Params, hidden, W, targets, lse, grad_coef, grad_loss=None, d_hidden=None, d_W=None,
+                   workspace: Optional[torch.Tensor] = None):
+    """ulorl_token_loss_bwd on the current CUDA stream.  Returns (d_hidden, d_W)."""
+    lib = load_library()
+    dev = hidden.device
+    if d_hidden is None:
+        d_hidden = torch.empty_like(hidden)
+    if d_W is None:
+        d_W = torch.zeros(p.V, p.H, dtype=torch.float32, device=dev) if p.dw_accumulate else \
+            torch.empty(p.V, p.H, dtype=torch.float32, device=dev)
+    _want(d_W, torch.float32, p.V * p.H, "d_W")
+    workspace = workspace if workspace is not None else alloc_workspace(p, dev)
+    code = lib.ulorl_token_loss_bwd(
+        ctypes.byref(p.to_c()), _ptr(hidden), _ptr(W), _ptr(targets), _ptr(lse), _ptr(grad_coef), _ptr(grad_loss),
+        _ptr(d_hidden), _ptr(d_W), _ptr(workspace), workspace.numel(), _stream())
+    _check(code, "ulorl_token_loss_bwd")
+    return d_hidden, d_W
+
+
+def check_status(workspace: torch.Tensor) -> int:
+    return int(load_library().ulorl_check_status(_ptr(workspace), _stream()))

@@ -1,0 +1,39 @@
+// Shared host/device definitions of the UloRL token-loss library.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ulorl.h"
+
+namespace ulorl {
+
+constexpr int kPartialStride = 4;   // floats per (token, vocab split): running max, sum exp, sum exp*z, pad
+constexpr int kMaxSplits = 32;
+
+// Device status word (first int of the workspace).  Bits, so that several problems can be kept.
+constexpr int kStatusTimeout = 1;
+constexpr int kStatusBadTarget = 2;
+
+// Per-block partial results of the decision kernel, reduced in block order by a final kernel
+// so that the loss and the statistics do not depend on scheduling.
+struct DecidePartial {
+  double loss_sum;
+  double stale_abs[ULORL_N_STALENESS];
+  int n_active, n_mpt, n_masked, n_clip_high, n_clip_low, pad;
+  int stale_tokens[ULORL_N_STALENESS];
+  int stale_clipped[ULORL_N_STALENESS];
+};
+
+// Values the host derives once per call for the decision stage.  The thresholds are float32
+// roundings of float64 evaluations, so that no transcendental sits inside a comparison.
+struct DecideConsts {
+  float ln_tau, ln_hi, ln_lo, sigma;
+  double eps_lo, eps_hi, inv_N;
+  int is_mode, mpt_mode, ent_scope, adv_per_token, current_version;
+};
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace ulorl

@@ -1,0 +1,249 @@
+// Per-token kernels after the LM-head pass: merge of the vocabulary splits, per-sequence mean
+// entropy, and the decision stage (ratio, mask, clipped surrogate, loss, d loss / d logp).
+#pragma once
+
+#include "common.cuh"
+
+namespace ulorl {
+
+// ------------------------------------------------------------------------------------------
+// Merge of the online-softmax partials of the vocabulary splits (log-softmax of Eq. 6, entropy
+// of Eq. 10).  partials[split][t] = (m, s, u, -) with m the running max of the raw accumulator
+// a = hidden . W[v], s = sum_v exp(kappa (a_v - m)), u = sum_v exp(kappa (a_v - m)) a_v.
+//   lse = kappa m* + ln s*,  logp = kappa a_y - lse,  Hent = lse - kappa u* / s*.
+// ------------------------------------------------------------------------------------------
+__global__ void merge_splits_kernel(int T, int n_split, float kappa, const float4* __restrict__ partials,
+                                    const float* __restrict__ acc_y, float* __restrict__ logp,
+                                    float* __restrict__ entropy, float* __restrict__ lse) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= T) return;
+  float m = -INFINITY;
+  for (int k = 0; k < n_split; ++k) m = fmaxf(m, partials[(size_t)k * T + t].x);
+  float s = 0.f, u = 0.f;
+  for (int k = 0; k < n_split; ++k) {
+    const float4 p = partials[(size_t)k * T + t];
+    if (p.x == -INFINITY) continue;
+    const float w = __expf(kappa * (p.x - m));
+    s = fmaf(p.y, w, s);
+    u = fmaf(p.z, w, u);
+  }
+  const float l = fmaf(kappa, m, logf(s));
+  if (lse) lse[t] = l;
+  if (logp) logp[t] = fmaf(kappa, acc_y[t], -l);
+  if (entropy) entropy[t] = fmaxf(l - kappa * u / s, 0.f);
+}
+
+// ------------------------------------------------------------------------------------------
+// H-bar_i of Eq. 10: mean per-token entropy of each sequence.  One block per sequence, float64
+// accumulation in a fixed order (thread-strided partial sums, then a fixed tree).
+// ------------------------------------------------------------------------------------------
+constexpr int kSeqThreads = 256;
+
+__global__ void seq_entropy_kernel(int S, const int* __restrict__ seq_offsets, const float* __restrict__ entropy,
+                                   double* __restrict__ seq_sum, float* __restrict__ seq_entropy) {
+  __shared__ double red[kSeqThreads];
+  const int i = blockIdx.x;
+  const int a = seq_offsets[i], b = seq_offsets[i + 1];
+  double acc = 0.0;
+  for (int t = a + threadIdx.x; t < b; t += kSeqThreads) acc += (double)entropy[t];
+  red[threadIdx.x] = acc;
+  __syncthreads();
+  for (int w = kSeqThreads / 2; w > 0; w >>= 1) {
+    if (threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    seq_sum[i] = red[0];
+    if (seq_entropy) seq_entropy[i] = b > a ? (float)(red[0] / (double)(b - a)) : 0.f;
+  }
+}
+
+// Token mean of the entropy over the whole call: the sequence sums added in sequence order.
+__global__ void batch_entropy_kernel(int S, int T, const double* __restrict__ seq_sum, float* __restrict__ batch_mean) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    double tot = 0.0;
+    for (int i = 0; i < S; ++i) tot += seq_sum[i];
+    *batch_mean = T > 0 ? (float)(tot / (double)T) : 0.f;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Decision stage, one token per thread.
+//   MPT (Eq. 9):        A > 0 and logp >= ln tau          gate (Eq. 10): H-bar < sigma
+//   ratio (Eq. 8):      d = logp - old_logp, r = exp(d)   (POIS: r = 1, nothing clipped)
+//   surrogate (Eq. 10): s = min(r A, clip(r, 1 - eps_lo, 1 + eps_hi) A)
+//   gradient:           g = -(1/N) (1 - msk) A r [not clipped]
+// Decisions are float32 comparisons against host-computed thresholds; values are float64.
+// ------------------------------------------------------------------------------------------
+constexpr int kDecideThreads = 256;
+
+__device__ __forceinline__ int find_sequence(const int* __restrict__ seq_offsets, int S, int t) {
+  int lo = 0, hi = S;   // largest i with seq_offsets[i] <= t
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (seq_offsets[mid] <= t) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+__global__ void decide_kernel(int T, int S, DecideConsts c, const float* __restrict__ logp,
+                              const float* __restrict__ old_logp, const int* __restrict__ segment_version,
+                              const float* __restrict__ advantages, const int* __restrict__ seq_offsets,
+                              const float* __restrict__ gate_entropy, const float* __restrict__ batch_mean,
+                              float* __restrict__ grad_coef, uint8_t* __restrict__ flags,
+                              DecidePartial* __restrict__ partials) {
+  __shared__ double sh_loss[kDecideThreads];
+  __shared__ float sh_abs[kDecideThreads];
+  __shared__ int sh_bucket[kDecideThreads];
+  __shared__ int sh_cnt[5];
+  __shared__ int sh_stale[2][ULORL_N_STALENESS];
+  const int tid = threadIdx.x;
+  const int t = blockIdx.x * kDecideThreads + tid;
+  if (tid < 5) sh_cnt[tid] = 0;
+  if (tid < ULORL_N_STALENESS) { sh_stale[0][tid] = 0; sh_stale[1][tid] = 0; }
+  __syncthreads();
+
+  double contrib = 0.0;
+  float dabs = 0.f;
+  int bucket = -1;
+  if (t < T) {
+    const int i = find_sequence(seq_offsets, S, t);
+    const float A = c.adv_per_token ? advantages[t] : advantages[i];
+    bool gate = false;
+    if (c.mpt_mode == ULORL_MPT_ALWAYS) {
+      gate = true;
+    } else if (c.mpt_mode == ULORL_MPT_DYNAMIC) {
+      const float h = (c.ent_scope == ULORL_ENT_BATCH) ? *batch_mean : gate_entropy[i];
+      gate = h < c.sigma;
+    }
+    const float lp = logp[t];
+    const bool mpt = (A > 0.f) && (lp >= c.ln_tau);
+    const bool msk = mpt && gate;
+    double r = 1.0;
+    bool hi = false, lo = false;
+    if (c.is_mode == ULORL_IS_SAIS) {
+      const float d = __fsub_rn(lp, old_logp[t]);
+      r = exp((double)d);
+      hi = (A > 0.f) && (d > c.ln_hi);
+      lo = (A < 0.f) && (d < c.ln_lo);
+      dabs = fabsf(d);
+    }
+    const double Ad = (double)A;
+    const double cl = fmin(fmax(r, 1.0 - c.eps_lo), 1.0 + c.eps_hi);
+    const double s = fmin(r * Ad, cl * Ad);
+    if (!msk) contrib = s;
+    const double g = (msk || hi || lo) ? 0.0 : -c.inv_N * Ad * r;
+    const float g32 = (float)g;
+    if (grad_coef) grad_coef[t] = g32;
+    const unsigned f = (msk ? ULORL_FLAG_MASKED : 0u) | (hi ? ULORL_FLAG_CLIP_HIGH : 0u) |
+                       (lo ? ULORL_FLAG_CLIP_LOW : 0u) | (mpt ? ULORL_FLAG_MPT : 0u);
+    if (flags) flags[t] = (uint8_t)f;
+    int st = segment_version ? c.current_version - segment_version[t] : 0;
+    st = st < 0 ? 0 : (st > ULORL_N_STALENESS - 1 ? ULORL_N_STALENESS - 1 : st);
+    bucket = st;
+    if (g != 0.0) atomicAdd(&sh_cnt[0], 1);
+    if (mpt) atomicAdd(&sh_cnt[1], 1);
+    if (msk) atomicAdd(&sh_cnt[2], 1);
+    if (hi) atomicAdd(&sh_cnt[3], 1);
+    if (lo) atomicAdd(&sh_cnt[4], 1);
+    atomicAdd(&sh_stale[0][st], 1);
+    if (hi || lo) atomicAdd(&sh_stale[1][st], 1);
+  }
+  sh_loss[tid] = contrib;
+  sh_abs[tid] = dabs;
+  sh_bucket[tid] = bucket;
+  __syncthreads();
+  for (int w = kDecideThreads / 2; w > 0; w >>= 1) {
+    if (tid < w) sh_loss[tid] += sh_loss[tid + w];
+    __syncthreads();
+  }
+  DecidePartial* out = partials + blockIdx.x;
+  if (tid < ULORL_N_STALENESS) {
+    double a = 0.0;
+    for (int k = 0; k < kDecideThreads; ++k)
+      if (sh_bucket[k] == tid) a += (double)sh_abs[k];
+    out->stale_abs[tid] = a;
+    out->stale_tokens[tid] = sh_stale[0][tid];
+    out->stale_clipped[tid] = sh_stale[1][tid];
+  }
+  if (tid == 0) {
+    out->loss_sum = sh_loss[0];
+    out->n_active = sh_cnt[0];
+    out->n_mpt = sh_cnt[1];
+    out->n_masked = sh_cnt[2];
+    out->n_clip_high = sh_cnt[3];
+    out->n_clip_low = sh_cnt[4];
+    out->pad = 0;
+  }
+}
+
+// Sum of the per-block partials in a fixed order; writes the loss and the statistics.
+constexpr int kFinalThreads = 256;
+
+template <typename V>
+__device__ __forceinline__ V block_sum_fixed(V v, V* sh) {
+  sh[threadIdx.x] = v;
+  __syncthreads();
+  for (int w = kFinalThreads / 2; w > 0; w >>= 1) {
+    if (threadIdx.x < w) sh[threadIdx.x] += sh[threadIdx.x + w];
+    __syncthreads();
+  }
+  V r = sh[0];
+  __syncthreads();
+  return r;
+}
+
+__global__ void finalize_kernel(int T, int n_blocks, double inv_N, const DecidePartial* __restrict__ partials,
+                                const float* __restrict__ batch_mean, const int* __restrict__ status,
+                                float* __restrict__ loss, ulorl_stats_t* __restrict__ stats) {
+  __shared__ double shd[kFinalThreads];
+  __shared__ int shi[kFinalThreads];
+  const int tid = threadIdx.x;
+  double l = 0.0;
+  int cnt[5] = {0, 0, 0, 0, 0};
+  for (int b = tid; b < n_blocks; b += kFinalThreads) {
+    l += partials[b].loss_sum;
+    cnt[0] += partials[b].n_active;
+    cnt[1] += partials[b].n_mpt;
+    cnt[2] += partials[b].n_masked;
+    cnt[3] += partials[b].n_clip_high;
+    cnt[4] += partials[b].n_clip_low;
+  }
+  const double loss_sum = block_sum_fixed<double>(l, shd);
+  int tot[5];
+  for (int k = 0; k < 5; ++k) tot[k] = block_sum_fixed<int>(cnt[k], shi);
+  const float loss_value = (float)(-loss_sum * inv_N);
+  if (tid == 0 && loss) loss[0] = loss_value;
+  if (!stats) return;
+  for (int s = 0; s < ULORL_N_STALENESS; ++s) {
+    double a = 0.0;
+    int nt = 0, nc = 0;
+    for (int b = tid; b < n_blocks; b += kFinalThreads) {
+      a += partials[b].stale_abs[s];
+      nt += partials[b].stale_tokens[s];
+      nc += partials[b].stale_clipped[s];
+    }
+    const double at = block_sum_fixed<double>(a, shd);
+    const int ntt = block_sum_fixed<int>(nt, shi);
+    const int nct = block_sum_fixed<int>(nc, shi);
+    if (tid == 0) {
+      stats->stale_tokens[s] = ntt;
+      stats->stale_clipped[s] = nct;
+      stats->stale_mean_abs_logratio[s] = ntt > 0 ? (float)(at / (double)ntt) : 0.f;
+    }
+  }
+  if (tid == 0) {
+    stats->loss = loss_value;
+    stats->mean_entropy = *batch_mean;
+    stats->n_tokens = T;
+    stats->n_active = tot[0];
+    stats->n_mpt = tot[1];
+    stats->n_masked = tot[2];
+    stats->n_clip_high = tot[3];
+    stats->n_clip_low = tot[4];
+    stats->device_status = *status;
+    stats->reserved[0] = stats->reserved[1] = stats->reserved[2] = 0;
+  }
+}
+
+}  // namespace ulorl

@@ -1,0 +1,473 @@
+// C ABI of the UloRL token-loss library: argument validation, workspace carve-up, tensor-map
+// construction and kernel launches.  No allocation, no synchronisation (except
+// ulorl_check_status), no state between calls.
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+
+#include "common.cuh"
+#include "elementwise.cuh"
+#include "simt.cuh"
+#include "umma_gemm.cuh"
+
+namespace ulorl {
+
+static std::atomic<long long> g_launches{0};
+constexpr int kDesignSMs = 148;           // the plan (splits, workspace) is sized for a B200
+constexpr int kDefaultPanelTensor = 16384;
+constexpr int kDefaultPanelSimt = 1024;
+
+struct Plan {
+  bool tensor;            // tensor-core path (bf16) or SIMT path
+  int n_split, tiles_per_split;
+  int panel_tokens;
+  size_t dz_ld;           // leading dimension of the dz panel (elements)
+  size_t off_status, off_batch_mean, off_seq_sum, off_partials, off_acc_y, off_decide, off_dz, total;
+  int decide_blocks;
+};
+
+static bool use_tensor_path(const ulorl_params_t* p) {
+  if (p->kernel_path == ULORL_PATH_SIMT) return false;
+  return p->dtype == ULORL_BF16;
+}
+
+static int validate_params(const ulorl_params_t* p) {
+  if (!p) return ULORL_ERR_INVALID_ARG;
+  if (p->T < 0 || p->H <= 0 || p->V <= 0 || p->num_seqs < 0) return ULORL_ERR_INVALID_ARG;
+  if (p->T > 0 && p->num_seqs == 0) return ULORL_ERR_INVALID_ARG;
+  if (p->dtype != ULORL_F32 && p->dtype != ULORL_BF16) return ULORL_ERR_UNSUPPORTED;
+  if (p->is_mode != ULORL_IS_SAIS && p->is_mode != ULORL_IS_POIS) return ULORL_ERR_INVALID_ARG;
+  if (p->mpt_mode < ULORL_MPT_OFF || p->mpt_mode > ULORL_MPT_DYNAMIC) return ULORL_ERR_INVALID_ARG;
+  if (p->ent_scope < ULORL_ENT_PER_SEQ || p->ent_scope > ULORL_ENT_SUPPLIED) return ULORL_ERR_INVALID_ARG;
+  if (p->kernel_path < ULORL_PATH_AUTO || p->kernel_path > ULORL_PATH_TENSOR) return ULORL_ERR_INVALID_ARG;
+  if (p->kernel_path == ULORL_PATH_TENSOR && p->dtype != ULORL_BF16) return ULORL_ERR_UNSUPPORTED;
+  if (!(p->inv_temperature > 0.f) || !std::isfinite(p->inv_temperature)) return ULORL_ERR_INVALID_ARG;
+  if (!(p->clip_eps_low >= 0.f) || !(p->clip_eps_high >= 0.f) || p->clip_eps_low > 1.f) return ULORL_ERR_INVALID_ARG;
+  if (!(p->mpt_tau > 0.f) || p->mpt_tau > 1.f) return ULORL_ERR_INVALID_ARG;
+  if (p->norm_tokens < 0 || p->bwd_panel_tokens < 0) return ULORL_ERR_INVALID_ARG;
+  if (p->H % 8 != 0) return ULORL_ERR_UNSUPPORTED;
+  return ULORL_OK;
+}
+
+static Plan make_plan(const ulorl_params_t* p) {
+  Plan pl{};
+  pl.tensor = use_tensor_path(p);
+  const int T = p->T, V = p->V;
+  const int tile_m = pl.tensor ? kBM : kSimtTile;
+  const int tile_n = pl.tensor ? kBN : kSimtTile;
+  const int m_tiles = (T + tile_m - 1) / tile_m;
+  const int n_tiles = (V + tile_n - 1) / tile_n;
+  int want = m_tiles > 0 ? (8 * kDesignSMs + m_tiles - 1) / m_tiles : 1;
+  want = want < 1 ? 1 : want;
+  want = want > kMaxSplits ? kMaxSplits : want;
+  want = want > n_tiles ? n_tiles : want;
+  pl.tiles_per_split = (n_tiles + want - 1) / want;
+  pl.n_split = (n_tiles + pl.tiles_per_split - 1) / pl.tiles_per_split;
+  int panel = p->bwd_panel_tokens > 0 ? p->bwd_panel_tokens : (pl.tensor ? kDefaultPanelTensor : kDefaultPanelSimt);
+  panel = (panel + kBM - 1) / kBM * kBM;
+  const int t_round = (T + kBM - 1) / kBM * kBM;
+  if (panel > t_round) panel = t_round;
+  if (panel < kBM) panel = kBM;
+  pl.panel_tokens = panel;
+  pl.dz_ld = pl.tensor ? align_up((size_t)V, 64) : (size_t)V;
+  pl.decide_blocks = (T + kDecideThreads - 1) / kDecideThreads;
+  size_t off = 0;
+  pl.off_status = off;      off += 256;
+  pl.off_batch_mean = pl.off_status + 16;
+  pl.off_seq_sum = off;     off = align_up(off + sizeof(double) * (size_t)(p->num_seqs > 0 ? p->num_seqs : 1), 256);
+  pl.off_partials = off;    off = align_up(off + sizeof(float4) * (size_t)pl.n_split * (size_t)(T > 0 ? T : 1), 256);
+  pl.off_acc_y = off;       off = align_up(off + sizeof(float) * (size_t)(T > 0 ? T : 1), 256);
+  pl.off_decide = off;      off = align_up(off + sizeof(DecidePartial) * (size_t)(pl.decide_blocks > 0 ? pl.decide_blocks : 1), 1024);
+  pl.off_dz = off;          off = align_up(off + (size_t)panel * pl.dz_ld * (pl.tensor ? 2 : 4), 1024);
+  pl.total = off;
+  return pl;
+}
+
+static int check_launch() {
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    std::fprintf(stderr, "ulorl: CUDA launch error: %s\n", cudaGetErrorString(e));
+    return ULORL_ERR_CUDA;
+  }
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return ULORL_OK;
+}
+
+#define ULORL_LAUNCH_CHECK()                    \
+  do {                                          \
+    const int _st = check_launch();             \
+    if (_st != ULORL_OK) return _st;            \
+  } while (0)
+
+// ------------------------------------------------------------------ tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// bf16 matrix [rows][cols] with `ld` elements between rows; box = box_cols x box_rows, 128-byte swizzle,
+// out-of-range elements read as zero.
+static int make_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
+                         uint32_t box_cols, uint32_t box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return ULORL_ERR_CUDA;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {ld * 2};
+  const cuuint32_t box[2] = {box_cols, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    std::fprintf(stderr, "ulorl: cuTensorMapEncodeTiled failed (%d)\n", (int)r);
+    return ULORL_ERR_CUDA;
+  }
+  return ULORL_OK;
+}
+
+template <int kMode>
+static int launch_umma(const CUtensorMap& ma, const CUtensorMap& mb, const UmmaArgs& a, cudaStream_t stream) {
+  static bool configured = false;
+  static int num_sms = 0;
+  if (!configured) {
+    if (cudaFuncSetAttribute(umma_kernel<kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUmmaSmemBytes) !=
+        cudaSuccess)
+      return ULORL_ERR_CUDA;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0)
+      return ULORL_ERR_CUDA;
+    configured = true;
+  }
+  const int units = (kMode == kModeStats) ? a.m_tiles * a.n_split : a.m_tiles * a.n_tiles;
+  if (units <= 0) return ULORL_OK;
+  const int grid = units < num_sms ? units : num_sms;
+  umma_kernel<kMode><<<grid, kUmmaThreads, kUmmaSmemBytes, stream>>>(ma, mb, a);
+  return check_launch();
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ------------------------------------------------------------------ decision stage
+static DecideConsts make_decide_consts(const ulorl_params_t* p) {
+  DecideConsts c{};
+  c.ln_tau = (float)std::log((double)p->mpt_tau);
+  c.ln_hi = (float)std::log1p((double)p->clip_eps_high);
+  c.ln_lo = p->clip_eps_low < 1.f ? (float)std::log1p(-(double)p->clip_eps_low) : -INFINITY;
+  c.sigma = p->entropy_target;
+  c.eps_lo = (double)p->clip_eps_low;
+  c.eps_hi = (double)p->clip_eps_high;
+  const double N = p->norm_tokens > 0 ? (double)p->norm_tokens : (double)p->T;
+  c.inv_N = N > 0 ? 1.0 / N : 0.0;
+  c.is_mode = p->is_mode;
+  c.mpt_mode = p->mpt_mode;
+  c.ent_scope = p->ent_scope;
+  c.adv_per_token = p->adv_per_token;
+  c.current_version = p->current_version;
+  return c;
+}
+
+static int run_decide(const ulorl_params_t* p, const Plan& pl, const float* logp, const float* entropy,
+                      const float* old_logp, const int32_t* segment_version, const float* advantages,
+                      const int32_t* seq_offsets, const float* entropy_supplied, float* grad_coef, uint8_t* flags,
+                      float* seq_entropy, float* loss, void* stats, uint8_t* ws, cudaStream_t stream) {
+  const int T = p->T, S = p->num_seqs;
+  int* status = reinterpret_cast<int*>(ws + pl.off_status);
+  float* batch_mean = reinterpret_cast<float*>(ws + pl.off_batch_mean);
+  double* seq_sum = reinterpret_cast<double*>(ws + pl.off_seq_sum);
+  DecidePartial* partials = reinterpret_cast<DecidePartial*>(ws + pl.off_decide);
+  // the gate needs a float array of per-sequence means even when the caller does not want it back
+  float* seq_ent_out = seq_entropy;
+  seq_entropy_kernel<<<S, kSeqThreads, 0, stream>>>(S, seq_offsets, entropy, seq_sum, seq_ent_out);
+  ULORL_LAUNCH_CHECK();
+  batch_entropy_kernel<<<1, 32, 0, stream>>>(S, T, seq_sum, batch_mean);
+  ULORL_LAUNCH_CHECK();
+  const DecideConsts c = make_decide_consts(p);
+  const float* gate = (p->ent_scope == ULORL_ENT_SUPPLIED) ? entropy_supplied : seq_ent_out;
+  decide_kernel<<<pl.decide_blocks, kDecideThreads, 0, stream>>>(T, S, c, logp, old_logp, segment_version, advantages,
+                                                                  seq_offsets, gate, batch_mean, grad_coef, flags,
+                                                                  partials);
+  ULORL_LAUNCH_CHECK();
+  finalize_kernel<<<1, kFinalThreads, 0, stream>>>(T, pl.decide_blocks, c.inv_N, partials, batch_mean, status, loss,
+                                                   reinterpret_cast<ulorl_stats_t*>(stats));
+  ULORL_LAUNCH_CHECK();
+  return ULORL_OK;
+}
+
+static int validate_decide_args(const ulorl_params_t* p, const float* old_logp, const float* advantages,
+                                const int32_t* seq_offsets, const float* entropy_supplied, float* seq_entropy,
+                                float* loss) {
+  if (!advantages || !seq_offsets || !loss || !seq_entropy) return ULORL_ERR_INVALID_ARG;
+  if (p->is_mode == ULORL_IS_SAIS && !old_logp) return ULORL_ERR_INVALID_ARG;
+  if (p->mpt_mode == ULORL_MPT_DYNAMIC && p->ent_scope == ULORL_ENT_SUPPLIED && !entropy_supplied)
+    return ULORL_ERR_INVALID_ARG;
+  return ULORL_OK;
+}
+
+// T == 0: nothing to compute; the loss and the statistics are zero.
+static int empty_forward(void* workspace, size_t workspace_bytes, float* loss, void* stats, cudaStream_t stream) {
+  if (!loss) return ULORL_ERR_INVALID_ARG;
+  if (workspace && workspace_bytes >= 256 && cudaMemsetAsync(workspace, 0, 256, stream) != cudaSuccess)
+    return ULORL_ERR_CUDA;
+  if (cudaMemsetAsync(loss, 0, sizeof(float), stream) != cudaSuccess) return ULORL_ERR_CUDA;
+  if (stats && cudaMemsetAsync(stats, 0, sizeof(ulorl_stats_t), stream) != cudaSuccess) return ULORL_ERR_CUDA;
+  return ULORL_OK;
+}
+
+}  // namespace ulorl
+
+using namespace ulorl;
+
+extern "C" {
+
+size_t ulorl_workspace_bytes(const ulorl_params_t* params) {
+  if (validate_params(params) != ULORL_OK) return 0;
+  return make_plan(params).total;
+}
+
+int64_t ulorl_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
+
+const char* ulorl_status_string(int status) {
+  switch (status) {
+    case ULORL_OK: return "ok";
+    case ULORL_ERR_INVALID_ARG: return "invalid argument";
+    case ULORL_ERR_UNSUPPORTED: return "unsupported shape, dtype or alignment";
+    case ULORL_ERR_WORKSPACE: return "workspace too small";
+    case ULORL_ERR_CUDA: return "CUDA call failed";
+    case ULORL_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+    case ULORL_ERR_BAD_TARGET: return "a target id was outside [0, V)";
+    default: return "unknown status";
+  }
+}
+
+int ulorl_check_status(void* workspace, void* cuda_stream) {
+  if (!workspace) return ULORL_ERR_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  int word = 0;
+  if (cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return ULORL_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return ULORL_ERR_CUDA;
+  if (word & kStatusTimeout) return ULORL_ERR_DEVICE_TIMEOUT;
+  if (word & kStatusBadTarget) return ULORL_ERR_BAD_TARGET;
+  return ULORL_OK;
+}
+
+int ulorl_token_loss_decide(const ulorl_params_t* params, const float* logp, const float* entropy,
+                            const float* old_logp, const int32_t* segment_version, const float* advantages,
+                            const int32_t* seq_offsets, const float* entropy_supplied, float* grad_coef,
+                            uint8_t* flags, float* seq_entropy, float* loss, void* stats, void* workspace,
+                            size_t workspace_bytes, void* cuda_stream) {
+  int st = validate_params(params);
+  if (st != ULORL_OK) return st;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (params->T == 0) return empty_forward(workspace, workspace_bytes, loss, stats, stream);
+  if (!logp || !entropy || !workspace) return ULORL_ERR_INVALID_ARG;
+  st = validate_decide_args(params, old_logp, advantages, seq_offsets, entropy_supplied, seq_entropy, loss);
+  if (st != ULORL_OK) return st;
+  const Plan pl = make_plan(params);
+  if (workspace_bytes < pl.total) return ULORL_ERR_WORKSPACE;
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  if (cudaMemsetAsync(ws + pl.off_status, 0, 256, stream) != cudaSuccess) return ULORL_ERR_CUDA;
+  return run_decide(params, pl, logp, entropy, old_logp, segment_version, advantages, seq_offsets, entropy_supplied,
+                    grad_coef, flags, seq_entropy, loss, stats, ws, stream);
+}
+
+int ulorl_token_loss_fwd(const ulorl_params_t* params, const void* hidden, const void* W, const int32_t* targets,
+                         const float* old_logp, const int32_t* segment_version, const float* advantages,
+                         const int32_t* seq_offsets, const float* entropy_supplied, float* logp, float* entropy,
+                         float* lse, float* grad_coef, uint8_t* flags, float* seq_entropy, float* loss, void* stats,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  int st = validate_params(params);
+  if (st != ULORL_OK) return st;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (params->T == 0) return empty_forward(workspace, workspace_bytes, loss, stats, stream);
+  if (!hidden || !W || !targets || !logp || !entropy || !lse || !workspace) return ULORL_ERR_INVALID_ARG;
+  st = validate_decide_args(params, old_logp, advantages, seq_offsets, entropy_supplied, seq_entropy, loss);
+  if (st != ULORL_OK) return st;
+  if (!aligned16(hidden) || !aligned16(W) || !aligned16(workspace)) return ULORL_ERR_UNSUPPORTED;
+  const Plan pl = make_plan(params);
+  if (workspace_bytes < pl.total) return ULORL_ERR_WORKSPACE;
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  const int T = params->T, H = params->H, V = params->V;
+  if (cudaMemsetAsync(ws + pl.off_status, 0, 256, stream) != cudaSuccess) return ULORL_ERR_CUDA;
+  int* status = reinterpret_cast<int*>(ws + pl.off_status);
+  float4* partials = reinterpret_cast<float4*>(ws + pl.off_partials);
+  float* acc_y = reinterpret_cast<float*>(ws + pl.off_acc_y);
+  const float kappa = params->inv_temperature;
+
+  if (pl.tensor) {
+    CUtensorMap map_a, map_b;
+    st = make_map_bf16(&map_a, hidden, (uint64_t)T, (uint64_t)H, (uint64_t)H, kBK, kBM);
+    if (st != ULORL_OK) return st;
+    st = make_map_bf16(&map_b, W, (uint64_t)V, (uint64_t)H, (uint64_t)H, kBK, kBN);
+    if (st != ULORL_OK) return st;
+    UmmaArgs a{};
+    a.M = T; a.N = V; a.K = H;
+    a.m_tiles = (T + kBM - 1) / kBM;
+    a.n_tiles = (V + kBN - 1) / kBN;
+    a.n_split = pl.n_split;
+    a.tiles_per_split = pl.tiles_per_split;
+    a.kappa = kappa;
+    a.targets = targets;
+    a.partials = partials;
+    a.acc_y = acc_y;
+    a.T_total = T;
+    a.status = status;
+    st = launch_umma<kModeStats>(map_a, map_b, a, stream);
+    if (st != ULORL_OK) return st;
+  } else {
+    const dim3 grid((T + kSimtTile - 1) / kSimtTile, pl.n_split);
+    if (params->dtype == ULORL_F32)
+      simt_stats_kernel<float><<<grid, kSimtThreads, 0, stream>>>(
+          static_cast<const float*>(hidden), static_cast<const float*>(W), targets, T, V, H, kappa, pl.tiles_per_split,
+          partials, acc_y, status);
+    else
+      simt_stats_kernel<__nv_bfloat16><<<grid, kSimtThreads, 0, stream>>>(
+          static_cast<const __nv_bfloat16*>(hidden), static_cast<const __nv_bfloat16*>(W), targets, T, V, H, kappa,
+          pl.tiles_per_split, partials, acc_y, status);
+    ULORL_LAUNCH_CHECK();
+  }
+  merge_splits_kernel<<<(T + 255) / 256, 256, 0, stream>>>(T, pl.n_split, kappa, partials, acc_y, logp, entropy, lse);
+  ULORL_LAUNCH_CHECK();
+  return run_decide(params, pl, logp, entropy, old_logp, segment_version, advantages, seq_offsets, entropy_supplied,
+                    grad_coef, flags, seq_entropy, loss, stats, ws, stream);
+}
+
+int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const void* W, const int32_t* targets,
+                         const float* lse, const float* grad_coef, const float* grad_loss, void* d_hidden, float* d_W,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  int st = validate_params(params);
+  if (st != ULORL_OK) return st;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const int T = params->T, H = params->H, V = params->V;
+  if (T == 0) {
+    if (!d_W) return ULORL_ERR_INVALID_ARG;
+    if (!params->dw_accumulate && cudaMemsetAsync(d_W, 0, sizeof(float) * (size_t)V * H, stream) != cudaSuccess)
+      return ULORL_ERR_CUDA;
+    return ULORL_OK;
+  }
+  if (!hidden || !W || !targets || !lse || !grad_coef || !d_hidden || !d_W || !workspace) return ULORL_ERR_INVALID_ARG;
+  if (!aligned16(hidden) || !aligned16(W) || !aligned16(d_hidden) || !aligned16(d_W) || !aligned16(workspace))
+    return ULORL_ERR_UNSUPPORTED;
+  const Plan pl = make_plan(params);
+  if (workspace_bytes < pl.total) return ULORL_ERR_WORKSPACE;
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  const float kappa = params->inv_temperature;
+  int* status = reinterpret_cast<int*>(ws + pl.off_status);
+
+  if (pl.tensor) {
+    __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(ws + pl.off_dz);
+    CUtensorMap map_hidden_k, map_w_k, map_w_mn, map_hidden_mn;
+    st = make_map_bf16(&map_hidden_k, hidden, (uint64_t)T, (uint64_t)H, (uint64_t)H, kBK, kBM);
+    if (st != ULORL_OK) return st;
+    st = make_map_bf16(&map_w_k, W, (uint64_t)V, (uint64_t)H, (uint64_t)H, kBK, kBN);
+    if (st != ULORL_OK) return st;
+    st = make_map_bf16(&map_w_mn, W, (uint64_t)V, (uint64_t)H, (uint64_t)H, 64, kBK);
+    if (st != ULORL_OK) return st;
+    st = make_map_bf16(&map_hidden_mn, hidden, (uint64_t)T, (uint64_t)H, (uint64_t)H, 64, kBK);
+    if (st != ULORL_OK) return st;
+    for (int t0 = 0, panel = 0; t0 < T; t0 += pl.panel_tokens, ++panel) {
+      const int rows = (T - t0) < pl.panel_tokens ? (T - t0) : pl.panel_tokens;
+      // dz panel: recompute logits, softmax minus one-hot scaled by the token's coefficient
+      {
+        UmmaArgs a{};
+        a.M = rows; a.N = V; a.K = H;
+        a.m_tiles = (rows + kBM - 1) / kBM;
+        a.n_tiles = (int)(pl.dz_ld / kBN) + ((pl.dz_ld % kBN) ? 1 : 0);
+        a.a_mn0 = t0;
+        a.row0 = t0;
+        a.kappa = kappa;
+        a.targets = targets; a.lse = lse; a.grad_coef = grad_coef; a.grad_loss = grad_loss;
+        a.dz = dz; a.dz_ld = pl.dz_ld; a.dz_cols = (int)pl.dz_ld;
+        a.status = status;
+        st = launch_umma<kModeDz>(map_hidden_k, map_w_k, a, stream);
+        if (st != ULORL_OK) return st;
+      }
+      CUtensorMap map_dz_k, map_dz_mn;
+      st = make_map_bf16(&map_dz_k, dz, (uint64_t)rows, (uint64_t)pl.dz_ld, (uint64_t)pl.dz_ld, kBK, kBM);
+      if (st != ULORL_OK) return st;
+      st = make_map_bf16(&map_dz_mn, dz, (uint64_t)rows, (uint64_t)pl.dz_ld, (uint64_t)pl.dz_ld, 64, kBK);
+      if (st != ULORL_OK) return st;
+      // d_hidden[t0 + m, h] = sum_v dz[m, v] W[v, h]
+      {
+        UmmaArgs a{};
+        a.M = rows; a.N = H; a.K = V;
+        a.m_tiles = (rows + kBM - 1) / kBM;
+        a.n_tiles = (H + kBN - 1) / kBN;
+        a.row0 = t0;
+        a.d_hidden = static_cast<__nv_bfloat16*>(d_hidden);
+        a.out_ld = (size_t)H;
+        a.status = status;
+        st = launch_umma<kModeDHidden>(map_dz_k, map_w_mn, a, stream);
+        if (st != ULORL_OK) return st;
+      }
+      // d_W[v, h] (+)= sum_m dz[m, v] hidden[t0 + m, h]
+      {
+        UmmaArgs a{};
+        a.M = V; a.N = H; a.K = rows;
+        a.m_tiles = (V + kBM - 1) / kBM;
+        a.n_tiles = (H + kBN - 1) / kBN;
+        a.b_k0 = t0;
+        a.d_W = d_W;
+        a.out_ld = (size_t)H;
+        a.accumulate = (panel > 0 || params->dw_accumulate) ? 1 : 0;
+        a.status = status;
+        st = launch_umma<kModeDW>(map_dz_mn, map_hidden_mn, a, stream);
+        if (st != ULORL_OK) return st;
+      }
+    }
+    return ULORL_OK;
+  }
+
+  // SIMT path: float32 dz panel, three CUDA-core contractions
+  float* dz = reinterpret_cast<float*>(ws + pl.off_dz);
+  for (int t0 = 0, panel = 0; t0 < T; t0 += pl.panel_tokens, ++panel) {
+    const int rows = (T - t0) < pl.panel_tokens ? (T - t0) : pl.panel_tokens;
+    const dim3 gdz((rows + kSimtTile - 1) / kSimtTile, (V + kSimtTile - 1) / kSimtTile);
+    const dim3 gdh((H + kSimtTile - 1) / kSimtTile, (rows + kSimtTile - 1) / kSimtTile);
+    const dim3 gdw((H + kSimtTile - 1) / kSimtTile, (V + kSimtTile - 1) / kSimtTile);
+    const int acc = (panel > 0 || params->dw_accumulate) ? 1 : 0;
+    if (params->dtype == ULORL_F32) {
+      const float* h = static_cast<const float*>(hidden);
+      const float* w = static_cast<const float*>(W);
+      simt_dz_kernel<float><<<gdz, kSimtThreads, 0, stream>>>(h, w, targets, lse, grad_coef, grad_loss, T, V, H, kappa,
+                                                               t0, t0 + rows, dz, pl.dz_ld);
+      ULORL_LAUNCH_CHECK();
+      simt_gemm_kernel<float, float, float><<<gdh, kSimtThreads, 0, stream>>>(
+          dz, pl.dz_ld, 1, w, (size_t)H, 1, static_cast<float*>(d_hidden) + (size_t)t0 * H, (size_t)H, rows, H, V, 0);
+      ULORL_LAUNCH_CHECK();
+      simt_gemm_kernel<float, float, float><<<gdw, kSimtThreads, 0, stream>>>(
+          dz, 1, pl.dz_ld, h + (size_t)t0 * H, (size_t)H, 1, d_W, (size_t)H, V, H, rows, acc);
+      ULORL_LAUNCH_CHECK();
+    } else {
+      const __nv_bfloat16* h = static_cast<const __nv_bfloat16*>(hidden);
+      const __nv_bfloat16* w = static_cast<const __nv_bfloat16*>(W);
+      simt_dz_kernel<__nv_bfloat16><<<gdz, kSimtThreads, 0, stream>>>(h, w, targets, lse, grad_coef, grad_loss, T, V, H,
+                                                                       kappa, t0, t0 + rows, dz, pl.dz_ld);
+      ULORL_LAUNCH_CHECK();
+      simt_gemm_kernel<float, __nv_bfloat16, __nv_bfloat16><<<gdh, kSimtThreads, 0, stream>>>(
+          dz, pl.dz_ld, 1, w, (size_t)H, 1, static_cast<__nv_bfloat16*>(d_hidden) + (size_t)t0 * H, (size_t)H, rows, H,
+          V, 0);
+      ULORL_LAUNCH_CHECK();
+      simt_gemm_kernel<float, __nv_bfloat16, float><<<gdw, kSimtThreads, 0, stream>>>(
+          dz, 1, pl.dz_ld, h + (size_t)t0 * H, (size_t)H, 1, d_W, (size_t)H, V, H, rows, acc);
+      ULORL_LAUNCH_CHECK();
+    }
+  }
+  return ULORL_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,386 @@
+// Tensor-core kernels (tcgen05 / tensor memory / TMA) for the four dense contractions of the
+// token-loss path, bf16 inputs and float32 accumulation:
+//
+//   kModeStats   a = hidden . W^T per (token tile, vocabulary tile); the epilogue reduces the tile to
+//                online-softmax statistics per token (Eq. 6, Eq. 10) -- logits never leave the SM
+//   kModeDz      same contraction, epilogue writes dz = coef * (onehot - softmax) as bf16 to a token panel
+//   kModeDHidden d_hidden[t, :] = sum_v dz[t, v] W[v, :]
+//   kModeDW      d_W[v, :] (+)= sum_t dz[t, v] hidden[t, :]
+//
+// One persistent CTA per SM, 192 threads: warp 0 feeds a 4-stage shared-memory ring with TMA tile
+// loads (128-byte swizzle), warp 1 issues tcgen05.mma (128 x 256 x 16 per instruction) into one of
+// two 256-column tensor-memory accumulators, warps 2-5 drain the other accumulator with tcgen05.ld
+// (one token row per thread) and run the mode's epilogue, so the epilogue of tile i overlaps the
+// contraction of tile i + 1.  Operands whose contraction index is not the contiguous one in memory
+// (W and hidden in the two gradient contractions, dz in the d_W one) are loaded as MN-major tiles;
+// nothing is transposed in global memory.
+#pragma once
+
+#include "common.cuh"
+#include "ptx_sm100.cuh"
+
+namespace ulorl {
+
+constexpr int kBM = 128;           // accumulator rows (tensor-memory lanes)
+constexpr int kBN = 256;           // accumulator columns
+constexpr int kBK = 64;            // contraction elements per pipeline stage (128 bytes of bf16)
+constexpr int kUmmaK = 16;         // contraction elements per tcgen05.mma
+constexpr int kStages = 4;
+constexpr int kUmmaThreads = 192;
+constexpr int kTmemCols = 512;     // two accumulators of kBN columns
+constexpr uint32_t kABytes = kBM * kBK * 2;
+constexpr uint32_t kBBytes = kBN * kBK * 2;
+constexpr uint32_t kStageBytes = kABytes + kBBytes;
+constexpr uint32_t kChunkBytes = 64 * kBK * 2;   // one MN-major box: 64 k-rows of 64 contiguous elements
+constexpr size_t kUmmaSmemBytes = (size_t)kStages * kStageBytes + 1024;
+constexpr long long kWaitLimitCycles = 4000000000LL;   // about two seconds at the maximum SM clock
+
+enum UmmaMode { kModeStats = 0, kModeDz = 1, kModeDHidden = 2, kModeDW = 3 };
+
+struct UmmaArgs {
+  int M, N, K;              // extents of the contraction handled by this launch (valid elements)
+  int m_tiles, n_tiles;     // ceil(M / kBM), ceil(N / kBN)
+  int n_split;              // kModeStats: vocabulary splits; a unit is (token tile, split)
+  int tiles_per_split;
+  int a_mn0, a_k0;          // coordinate offsets of operand A in its tensor map (MN index, K index)
+  int b_mn0, b_k0;
+  int row0;                 // global token (or vocabulary row) index of accumulator row 0 of tile 0
+  float kappa;
+  const int* targets;
+  const float* lse;
+  const float* grad_coef;
+  const float* grad_loss;
+  float4* partials;         // kModeStats: [n_split][T_total]
+  float* acc_y;             // kModeStats: raw accumulator at the target column, [T_total]
+  int T_total;
+  __nv_bfloat16* dz;        // kModeDz: panel [rows][dz_ld]
+  size_t dz_ld;
+  int dz_cols;              // kModeDz: columns to write per row (>= N, zero beyond N)
+  __nv_bfloat16* d_hidden;  // kModeDHidden: [T][out_ld]
+  float* d_W;               // kModeDW: [V][out_ld]
+  size_t out_ld;
+  int accumulate;
+  int* status;
+};
+
+template <int kMode>
+struct ModeTraits {
+  static constexpr bool a_mn = (kMode == kModeDW);
+  static constexpr bool b_mn = (kMode == kModeDHidden || kMode == kModeDW);
+};
+
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+template <int kMode>
+__global__ void __launch_bounds__(kUmmaThreads, 1)
+umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const UmmaArgs args) {
+  using namespace ptx;
+  constexpr bool kAmn = ModeTraits<kMode>::a_mn;
+  constexpr bool kBmn = ModeTraits<kMode>::b_mn;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bar_full[kStages];
+  __shared__ __align__(8) uint64_t bar_empty[kStages];
+  __shared__ __align__(8) uint64_t bar_tmem_full[2];
+  __shared__ __align__(8) uint64_t bar_tmem_empty[2];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  volatile int* abort_p = &abort_flag;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(smem_u32(&bar_full[s]), 1);
+      mbar_init(smem_u32(&bar_empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bar_tmem_full[b]), 1);
+      mbar_init(smem_u32(&bar_tmem_empty[b]), 4);   // one arrival per epilogue warp
+    }
+    mbar_fence_init();
+    fence_async_proxy();
+  }
+  if (warp == 0 && lane == 0) {
+    prefetch_tensormap(&map_a);
+    prefetch_tensormap(&map_b);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&tmem_base_slot), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  const int k_blocks = (args.K + kBK - 1) / kBK;
+  const int n_units = (kMode == kModeStats) ? args.m_tiles * args.n_split : args.m_tiles * args.n_tiles;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    uint32_t stage = 0, phase = 0;
+    uint32_t issued = 0;
+    for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+      int m_tile, n_begin, n_end;
+      if (kMode == kModeStats) {
+        m_tile = unit / args.n_split;
+        n_begin = (unit % args.n_split) * args.tiles_per_split;
+        n_end = min(args.n_tiles, n_begin + args.tiles_per_split);
+      } else {
+        m_tile = unit / args.n_tiles;
+        n_begin = unit % args.n_tiles;
+        n_end = n_begin + 1;
+      }
+      for (int n_tile = n_begin; n_tile < n_end; ++n_tile) {
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait_bounded(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p, kWaitLimitCycles)) goto producer_drain;
+          if (lane == 0) {
+            const uint32_t full = smem_u32(&bar_full[stage]);
+            const uint32_t sa = smem_base + stage * kStageBytes;
+            const uint32_t sb = sa + kABytes;
+            mbar_arrive_expect_tx(full, kStageBytes);
+            if (kAmn) {
+#pragma unroll
+              for (int j = 0; j < kBM / 64; ++j)
+                tma_load_2d(sa + j * kChunkBytes, &map_a, full, args.a_mn0 + m_tile * kBM + j * 64, args.a_k0 + kb * kBK);
+            } else {
+              tma_load_2d(sa, &map_a, full, args.a_k0 + kb * kBK, args.a_mn0 + m_tile * kBM);
+            }
+            if (kBmn) {
+#pragma unroll
+              for (int j = 0; j < kBN / 64; ++j)
+                tma_load_2d(sb + j * kChunkBytes, &map_b, full, args.b_mn0 + n_tile * kBN + j * 64, args.b_k0 + kb * kBK);
+            } else {
+              tma_load_2d(sb, &map_b, full, args.b_k0 + kb * kBK, args.b_mn0 + n_tile * kBN);
+            }
+          }
+          __syncwarp();
+          ++issued;
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  producer_drain:
+    if (*abort_p) {
+      // give the copies still in flight a bounded time to land before the block goes away
+      const uint32_t n_back = issued < (uint32_t)kStages ? issued : (uint32_t)kStages;
+      for (uint32_t b = 0; b < n_back; ++b) {
+        if (stage == 0) { stage = kStages; phase ^= 1u; }
+        --stage;
+        const long long t0 = clock64();
+        while (!mbar_try_wait(smem_u32(&bar_full[stage]), phase) && clock64() - t0 < 200000000LL) {
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    constexpr uint32_t idesc = make_idesc_bf16(kBM, kBN, kAmn ? 1 : 0, kBmn ? 1 : 0);
+    uint32_t stage = 0, phase = 0;
+    uint32_t acc_iter = 0;
+    for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+      int n_begin, n_end;
+      if (kMode == kModeStats) {
+        n_begin = (unit % args.n_split) * args.tiles_per_split;
+        n_end = min(args.n_tiles, n_begin + args.tiles_per_split);
+      } else {
+        n_begin = 0;
+        n_end = 1;
+      }
+      for (int n_tile = n_begin; n_tile < n_end; ++n_tile, ++acc_iter) {
+        const uint32_t buf = acc_iter & 1u;
+        const uint32_t buf_phase = (acc_iter >> 1) & 1u;
+        if (!mbar_wait_bounded(smem_u32(&bar_tmem_empty[buf]), buf_phase ^ 1u, abort_p, kWaitLimitCycles)) goto role_done;
+        tc_fence_after_sync();
+        const uint32_t tmem_d = tmem_base + buf * kBN;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait_bounded(smem_u32(&bar_full[stage]), phase, abort_p, kWaitLimitCycles)) goto role_done;
+          tc_fence_after_sync();
+          if (lane == 0) {
+            const uint32_t sa = smem_base + stage * kStageBytes;
+            const uint32_t sb = sa + kABytes;
+#pragma unroll
+            for (int k = 0; k < kBK / kUmmaK; ++k) {
+              // K-major: 16 elements = 32 bytes along the swizzled row; MN-major: 16 k-rows of 128 bytes
+              const uint64_t da = kAmn ? make_smem_desc(sa + k * (kUmmaK * 128), kChunkBytes, 1024)
+                                       : make_smem_desc(sa + k * (kUmmaK * 2), 16, 1024);
+              const uint64_t db = kBmn ? make_smem_desc(sb + k * (kUmmaK * 128), kChunkBytes, 1024)
+                                       : make_smem_desc(sb + k * (kUmmaK * 2), 16, 1024);
+              umma_bf16(tmem_d, da, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            }
+            umma_commit(smem_u32(&bar_empty[stage]));                       // frees the smem slot
+            if (kb == k_blocks - 1) umma_commit(smem_u32(&bar_tmem_full[buf]));  // accumulator ready
+          }
+          __syncwarp();
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int quarter = warp & 3;                       // tensor-memory lanes 32 * quarter ..
+    const int row_in_tile = quarter * 32 + lane;
+    const float c2 = args.kappa * 1.4426950408889634f;  // exp(kappa a) = 2^(c2 a)
+    uint32_t acc_iter = 0;
+    for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+      int m_tile, n_begin, n_end, split = 0;
+      if (kMode == kModeStats) {
+        m_tile = unit / args.n_split;
+        split = unit % args.n_split;
+        n_begin = split * args.tiles_per_split;
+        n_end = min(args.n_tiles, n_begin + args.tiles_per_split);
+      } else {
+        m_tile = unit / args.n_tiles;
+        n_begin = unit % args.n_tiles;
+        n_end = n_begin + 1;
+      }
+      const int row = m_tile * kBM + row_in_tile;       // row within this launch's M extent
+      const bool row_ok = row < args.M;
+      const int grow = args.row0 + row;                 // global token / vocabulary row
+
+      // per-row state
+      float run_m = -INFINITY, run_s = 0.f, run_u = 0.f;
+      int y = -1;
+      float coef = 0.f, lse2 = 0.f;
+      if (kMode == kModeStats || kMode == kModeDz) {
+        if (row_ok) {
+          y = args.targets[grow];
+          if (y < 0 || y >= args.N) {
+            if (kMode == kModeStats) atomicOr(args.status, kStatusBadTarget);
+            y = y < 0 ? 0 : args.N - 1;
+          }
+        }
+      }
+      if (kMode == kModeDz) {
+        if (row_ok) {
+          const float gl = args.grad_loss ? *args.grad_loss : 1.f;
+          coef = args.kappa * gl * args.grad_coef[grow];
+          lse2 = args.lse[grow] * 1.4426950408889634f;
+        }
+      }
+
+      for (int n_tile = n_begin; n_tile < n_end; ++n_tile, ++acc_iter) {
+        const uint32_t buf = acc_iter & 1u;
+        const uint32_t buf_phase = (acc_iter >> 1) & 1u;
+        if (!mbar_wait_bounded(smem_u32(&bar_tmem_full[buf]), buf_phase, abort_p, kWaitLimitCycles)) goto role_done;
+        tc_fence_after_sync();
+        const uint32_t taddr = tmem_base + buf * kBN + ((uint32_t)(quarter * 32) << 16);
+        const int col_base = n_tile * kBN;
+#pragma unroll 1
+        for (int c = 0; c < kBN / 32; ++c) {
+          const int col0 = col_base + c * 32;
+          if (kMode != kModeDz && col0 >= args.N) break;       // whole chunk beyond the valid columns
+          if (kMode == kModeDz && col0 >= args.dz_cols) break;
+          uint32_t raw[32];
+          tmem_ld_32x32(taddr + c * 32, raw);
+          tmem_ld_wait();
+          const int nvalid = min(32, args.N - col0);           // may be <= 0 only in kModeDz padding
+
+          if (kMode == kModeStats) {
+            float cmax = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (j < nvalid) cmax = fmaxf(cmax, __uint_as_float(raw[j]));
+            const float m_new = fmaxf(run_m, cmax);
+            const float sc = ex2f((run_m - m_new) * c2);        // first chunk: 2^(-inf) = 0
+            run_s *= sc;
+            run_u *= sc;
+            run_m = m_new;
+            const float off = -m_new * c2;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              if (j < nvalid) {
+                const float a = __uint_as_float(raw[j]);
+                const float e = ex2f(fmaf(a, c2, off));
+                run_s += e;
+                run_u = fmaf(e, a, run_u);
+              }
+            }
+            if (row_ok && y >= col0 && y < col0 + 32) {
+              float ay = 0.f;
+#pragma unroll
+              for (int j = 0; j < 32; ++j) ay = (j == y - col0) ? __uint_as_float(raw[j]) : ay;
+              args.acc_y[grow] = ay;
+            }
+          } else if (kMode == kModeDz) {
+            uint32_t packed[16];
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+              float v0 = 0.f, v1 = 0.f;
+              if (j < nvalid) {
+                const float p = ex2f(fmaf(__uint_as_float(raw[j]), c2, -lse2));
+                v0 = coef * ((col0 + j == y ? 1.f : 0.f) - p);
+              }
+              if (j + 1 < nvalid) {
+                const float p = ex2f(fmaf(__uint_as_float(raw[j + 1]), c2, -lse2));
+                v1 = coef * ((col0 + j + 1 == y ? 1.f : 0.f) - p);
+              }
+              __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+              packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
+            }
+            if (row_ok) {
+              uint4* dst = reinterpret_cast<uint4*>(args.dz + (size_t)row * args.dz_ld + col0);
+              const int ncols = min(32, args.dz_cols - col0);     // multiple of 8
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+                if (q * 8 < ncols) dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+            }
+          } else if (kMode == kModeDHidden) {
+            if (row_ok) {
+              uint32_t packed[16];
+#pragma unroll
+              for (int j = 0; j < 32; j += 2) {
+                __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(raw[j]), __uint_as_float(raw[j + 1]));
+                packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
+              }
+              uint4* dst = reinterpret_cast<uint4*>(args.d_hidden + (size_t)grow * args.out_ld + col0);
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+                if (q * 8 < nvalid) dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+            }
+          } else {  // kModeDW
+            if (row_ok) {
+              float4* dst = reinterpret_cast<float4*>(args.d_W + (size_t)grow * args.out_ld + col0);
+#pragma unroll
+              for (int q = 0; q < 8; ++q) {
+                if (q * 4 < nvalid) {
+                  float4 v = make_float4(__uint_as_float(raw[4 * q]), __uint_as_float(raw[4 * q + 1]),
+                                         __uint_as_float(raw[4 * q + 2]), __uint_as_float(raw[4 * q + 3]));
+                  if (args.accumulate) {
+                    const float4 o = dst[q];
+                    v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+                  }
+                  dst[q] = v;
+                }
+              }
+            }
+          }
+        }
+        // accumulator drained: hand the buffer back to the MMA warp
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bar_tmem_empty[buf]));
+      }
+
+      if (kMode == kModeStats && row_ok)
+        args.partials[(size_t)split * args.T_total + grow] = make_float4(run_m, run_s, run_u, 0.f);
+    }
+  }
+
+role_done:
+  if (*abort_p && lane == 0) atomicOr(args.status, kStatusTimeout);
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace ulorl

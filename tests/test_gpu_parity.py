@@ -1,0 +1,319 @@
+"""Parity of the CUDA path (through the C ABI) against the fp64 oracle, element by element, on
+seeded workloads the oracle finishes in seconds.  Tolerances: log-prob and entropy 2e-3 abs,
+loss 1e-3 rel, gradients 1e-2 rel-L2; masks and clip flags exact on identical log-probs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ulorl_oracle as O
+from paper_2507_19766_b200 import binding as B
+from paper_2507_19766_b200 import synth
+from tests.helpers import TOL_GRAD, TOL_LOGP, TOL_LOSS, both_params, near_threshold, oracle_inputs, rel_l2
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+STAT_KEYS = ("n_tokens", "n_active", "n_mpt", "n_masked", "n_clip_high", "n_clip_low")
+
+
+def gpu_fwd_bwd(batch, gp, grad_loss=None, entropy_supplied=None):
+    b = batch.to(DEV)
+    ws = B.alloc_workspace(gp, DEV)
+    es = None if entropy_supplied is None else torch.tensor(entropy_supplied, dtype=torch.float32, device=DEV)
+    out = B.token_loss_fwd(gp, b.hidden, b.W, b.targets, b.old_logp, b.segment_version, b.advantages,
+                           b.seq_offsets, entropy_supplied=es, workspace=ws)
+    gl = None if grad_loss is None else torch.tensor([grad_loss], dtype=torch.float32, device=DEV)
+    dH, dW = B.token_loss_bwd(gp, b.hidden, b.W, b.targets, out.lse, out.grad_coef, grad_loss=gl, workspace=ws)
+    torch.cuda.synchronize()
+    assert B.check_status(ws) == B.OK
+    return out, dH, dW
+
+
+def check_against_oracle(batch, gp, op, grad_loss=None, check_grads=True):
+    out, dH, dW = gpu_fwd_bwd(batch, gp, grad_loss=grad_loss)
+    oi = oracle_inputs(batch)
+    ref = O.forward(oi["hidden"], oi["W"], oi["targets"], oi["old_logp"], oi["segment_version"], oi["advantages"],
+                    oi["seq_offsets"], op)
+    logp = out.logp.cpu().numpy()
+    ent = out.entropy.cpu().numpy()
+    lse = out.lse.cpu().numpy()
+    assert np.abs(logp - ref["logp"]).max() <= TOL_LOGP
+    assert np.abs(ent - ref["entropy"]).max() <= TOL_LOGP
+    assert np.abs(lse - ref["lse"]).max() <= TOL_LOGP
+    seq_ent = out.seq_entropy.cpu().numpy()[: batch.workload.S]
+    assert np.abs(seq_ent - ref["seq_entropy"]).max() <= TOL_LOGP
+
+    # decisions: exact wherever the oracle's own value is not within the tolerance of a threshold
+    flags = out.flags.cpu().numpy()
+    near = near_threshold(ref["logp"], oi["old_logp"], ref["seq_entropy"], oi["seq_offsets"], op)
+    differ = flags != ref["flags"]
+    assert not (differ & ~near).any(), f"{int((differ & ~near).sum())} decisions differ away from any threshold"
+
+    # decisions and values re-derived by the oracle from the GPU's own float32 log-probs: exact flags
+    gate = O.gate_entropy(ent, oi["seq_offsets"], op.ent_scope)
+    assert np.abs(gate - seq_ent).max() <= 1e-6 or op.ent_scope != "per_seq"
+    dec = O.decide(logp, seq_ent if op.ent_scope == "per_seq" else gate, oi["old_logp"], oi["advantages"],
+                   oi["seq_offsets"], oi["segment_version"], op)
+    assert np.array_equal(flags, dec["flags"])
+    g = out.grad_coef.cpu().numpy()
+    assert np.allclose(g, dec["grad_coef"], rtol=2e-6, atol=1e-12)
+    st = out.stats_host()
+    for k in STAT_KEYS:
+        assert st[k] == dec["stats"][k], k
+    assert st["stale_tokens"] == dec["stats"]["stale_tokens"].tolist()
+    assert st["stale_clipped"] == dec["stats"]["stale_clipped"].tolist()
+    assert np.allclose(st["stale_mean_abs_logratio"], dec["stats"]["stale_mean_abs_logratio"], rtol=1e-5, atol=1e-7)
+    assert st["device_status"] == 0
+    loss = float(out.loss.cpu()[0])
+    assert abs(loss - dec["loss"]) <= 2e-6 * max(1.0, abs(dec["loss"]))
+    if not differ.any():
+        assert abs(loss - ref["loss"]) <= TOL_LOSS * max(abs(ref["loss"]), 1e-3)
+    assert abs(st["mean_entropy"] - ref["mean_entropy"]) <= TOL_LOGP
+
+    if check_grads:
+        g_ref = dec["grad_coef"] if differ.any() else ref["grad_coef"]
+        dH_ref, dW_ref = O.backward(oi["hidden"], oi["W"], oi["targets"], g_ref, op.inv_temperature,
+                                    grad_loss=1.0 if grad_loss is None else grad_loss)
+        eh = rel_l2(dH.float().cpu().numpy(), dH_ref)
+        ew = rel_l2(dW.cpu().numpy(), dW_ref)
+        assert eh <= TOL_GRAD and ew <= TOL_GRAD, (eh, ew)
+        # sum_v dz[t, v] = 0, so the column sums of d_W vanish
+        col = np.abs(dW.double().sum(dim=0).cpu().numpy()).max()
+        assert col <= 1e-3 * max(1e-12, float(dW.abs().max()))
+    return out, ref
+
+
+# --------------------------------------------------------------------------- named workloads
+def test_tiny_f32():
+    wl = synth.WORKLOADS["tiny"]
+    batch = synth.make_batch(wl)
+    gp, op = both_params(batch)
+    out, ref = check_against_oracle(batch, gp, op)
+
+
+def test_tiny_f32_old_logp_from_oracle():
+    """The 'tiny' recipe as stated: old_logp = the oracle's current log-prob + N(0, 0.05)."""
+    wl = synth.WORKLOADS["tiny"]
+    b0 = synth.make_batch(wl)
+    oi = oracle_inputs(b0)
+    logp, _, _ = O.token_stats(oi["hidden"], oi["W"], oi["targets"])
+    batch = synth.make_batch(wl, base_logp=logp.astype(np.float32))
+    gp, op = both_params(batch)
+    check_against_oracle(batch, gp, op)
+
+
+@pytest.mark.parametrize("mpt_mode", ["always", "dynamic", "off"])
+def test_tiny_planted_mask_fires(mpt_mode):
+    wl = synth.WORKLOADS["tiny"].scaled(planted=0.5, beta_planted=(120.0, 220.0), mpt_mode=mpt_mode,
+                                        entropy_target=5.0)
+    batch = synth.make_batch(wl, seed=77)
+    gp, op = both_params(batch)
+    out, ref = check_against_oracle(batch, gp, op)
+    if mpt_mode != "off":
+        assert ref["stats"]["n_masked"] > 20
+    assert ref["stats"]["n_mpt"] > 20
+
+
+@pytest.mark.parametrize("path", ["tensor", "simt"])
+def test_bf16_mini_ragged(path):
+    """bf16, several token tiles with a ragged tail, vocabulary not a multiple of any tile width,
+    hidden size not a multiple of the 64-element pipeline stage, two backward panels."""
+    wl = synth.WORKLOADS["small"].scaled(T=700, S=5, H=328, V=3001, lengths="lognormal:100:400",
+                                         segment_len=64, planted=0.3, beta_planted=(80.0, 160.0),
+                                         mpt_mode="dynamic", entropy_target=6.0)
+    batch = synth.make_batch(wl, seed=5)
+    gp, op = both_params(batch, kernel_path=path, bwd_panel_tokens=384)
+    check_against_oracle(batch, gp, op)
+
+
+def test_bf16_temperature_and_grad_loss():
+    wl = synth.WORKLOADS["small"].scaled(T=512, S=4, H=256, V=2048, lengths="tiny", segment_len=100)
+    batch = synth.make_batch(wl, seed=9)
+    gp, op = both_params(batch, inv_temperature=1.0 / 0.85, norm_tokens=4096)
+    check_against_oracle(batch, gp, op, grad_loss=0.5)
+
+
+def test_small_bf16_full():
+    """The 'small' workload in full: T=16384, H=1024, V=32768 (oracle: tens of seconds)."""
+    wl = synth.WORKLOADS["small"]
+    batch = synth.make_batch(wl)
+    gp, op = both_params(batch)
+    check_against_oracle(batch, gp, op)
+
+
+def test_pois_path():
+    wl = synth.WORKLOADS["small"].scaled(T=640, S=6, H=256, V=4096, lengths="lognormal:100:300", segment_len=50,
+                                         is_mode="pois", planted=0.4, beta_planted=(100.0, 200.0), noise="stale:0.02",
+                                         mpt_mode="always")
+    batch = synth.make_batch(wl, seed=3)
+    gp, op = both_params(batch)
+    out, ref = check_against_oracle(batch, gp, op)
+    assert ref["stats"]["n_clip_high"] == 0 and ref["stats"]["n_clip_low"] == 0
+    # POIS does not read old_logp: NULL is accepted and gives the same result
+    b = batch.to(DEV)
+    out2 = B.token_loss_fwd(gp, b.hidden, b.W, b.targets, None, b.segment_version, b.advantages, b.seq_offsets)
+    assert torch.equal(out2.grad_coef, out.grad_coef) and torch.equal(out2.loss, out.loss)
+
+
+# --------------------------------------------------------------------------- tensor path vs SIMT path
+def test_tensor_path_matches_simt_path():
+    wl = synth.WORKLOADS["small"].scaled(T=1000, S=3, H=512, V=5000, lengths="lognormal:300:600", segment_len=128)
+    batch = synth.make_batch(wl, seed=21)
+    res = {}
+    for path in ("tensor", "simt"):
+        gp, _ = both_params(batch, kernel_path=path)
+        res[path] = gpu_fwd_bwd(batch, gp)
+    a, b = res["tensor"], res["simt"]
+    assert (a[0].logp - b[0].logp).abs().max() <= 1e-4
+    assert (a[0].entropy - b[0].entropy).abs().max() <= 1e-4
+    assert rel_l2(a[1].float().cpu().numpy(), b[1].float().cpu().numpy()) <= 1e-2
+    assert rel_l2(a[2].cpu().numpy(), b[2].cpu().numpy()) <= 1e-2
+
+
+# --------------------------------------------------------------------------- decision stage, bit exact
+@pytest.mark.parametrize("mode,mpt,scope", [("sais", "dynamic", "per_seq"), ("sais", "always", "per_seq"),
+                                            ("pois", "dynamic", "batch"), ("sais", "dynamic", "supplied"),
+                                            ("sais", "off", "per_seq")])
+def test_decide_bit_exact_on_oracle_logp(mode, mpt, scope):
+    """Feed the elementwise kernel the oracle's float32 log-probs and entropies: flags and counts
+    must match bit for bit, values to float32 rounding."""
+    rng = np.random.default_rng(12)
+    T, S = 5000, 7
+    cuts = np.sort(rng.choice(np.arange(1, T), size=S - 1, replace=False))
+    offsets = np.concatenate([[0], cuts, [T]]).astype(np.int32)
+    logp = (-np.abs(rng.standard_normal(T)) * 0.02).astype(np.float32)        # many tokens near ln(0.99)
+    logp[rng.random(T) < 0.3] -= np.float32(3.0)
+    ent = np.abs(rng.standard_normal(T)).astype(np.float32) * 0.25
+    old = (logp + rng.standard_normal(T).astype(np.float32) * 0.15).astype(np.float32)
+    adv = rng.choice(np.float32([1.0, -1.0, 0.0, 0.7]), size=S).astype(np.float32)
+    version = rng.integers(0, 9, size=T).astype(np.int32)
+    supplied = rng.random(S).astype(np.float32) * 0.4
+    kw = dict(is_mode=mode, mpt_mode=mpt, ent_scope=scope, entropy_target=0.2, current_version=8,
+              clip_eps_low=0.2, clip_eps_high=0.28)
+    op = O.OracleParams(**kw)
+    gp = B.Params(T=T, H=8, V=16, num_seqs=S, dtype="f32", **kw)
+    gate = O.gate_entropy(ent, offsets, scope, supplied)
+    ref = O.decide(logp, gate, old, adv, offsets, version, op)
+    t = lambda x: torch.from_numpy(x).to(DEV)
+    out = B.token_loss_decide(gp, t(logp), t(ent), t(old), t(version), t(adv), t(offsets),
+                              entropy_supplied=t(supplied))
+    torch.cuda.synchronize()
+    assert np.array_equal(out.flags.cpu().numpy(), ref["flags"])
+    st = out.stats_host()
+    for k in STAT_KEYS:
+        assert st[k] == ref["stats"][k], k
+    assert st["stale_tokens"] == ref["stats"]["stale_tokens"].tolist()
+    assert st["stale_clipped"] == ref["stats"]["stale_clipped"].tolist()
+    assert np.allclose(out.grad_coef.cpu().numpy(), ref["grad_coef"], rtol=1e-6, atol=0)
+    assert abs(float(out.loss.cpu()[0]) - ref["loss"]) <= 1e-6 * max(1.0, abs(ref["loss"]))
+    seq_mean, batch_mean = O.sequence_mean_entropy(ent, offsets)
+    assert np.allclose(out.seq_entropy.cpu().numpy()[:S], seq_mean, rtol=1e-6)
+    assert abs(st["mean_entropy"] - batch_mean) <= 1e-6
+    if mpt != "off":
+        assert ref["stats"]["n_masked"] > 0
+    if mode == "sais":
+        assert ref["stats"]["n_clip_high"] > 0 and ref["stats"]["n_clip_low"] > 0
+
+
+# --------------------------------------------------------------------------- edge cases
+def test_single_token_and_length_one_sequences():
+    wl = synth.WORKLOADS["small"].scaled(T=3, S=3, H=64, V=256, lengths="tiny", segment_len=1)
+    batch = synth.make_batch(wl, seed=2)
+    gp, op = both_params(batch)
+    check_against_oracle(batch, gp, op)
+    wl1 = synth.WORKLOADS["tiny"].scaled(T=1, S=1, H=64, V=100, lengths="single")
+    b1 = synth.make_batch(wl1, seed=4)
+    gp, op = both_params(b1)
+    check_against_oracle(b1, gp, op)
+
+
+def test_all_tokens_masked_gives_zero_loss_and_gradients():
+    wl = synth.WORKLOADS["small"].scaled(T=300, S=2, H=128, V=1024, lengths="tiny", planted=1.0,
+                                         beta_planted=(400.0, 500.0), adv="plus1", mpt_mode="always")
+    batch = synth.make_batch(wl, seed=6)
+    gp, op = both_params(batch)
+    out, dH, dW = gpu_fwd_bwd(batch, gp)
+    st = out.stats_host()
+    assert st["n_masked"] == 300 and st["n_active"] == 0
+    assert float(out.loss.cpu()[0]) == 0.0
+    assert float(dH.float().abs().max()) == 0.0 and float(dW.abs().max()) == 0.0
+
+
+def test_zero_advantage_sequences_contribute_nothing():
+    wl = synth.WORKLOADS["small"].scaled(T=256, S=4, H=128, V=512, lengths="tiny", adv="bern:0.0:4")
+    batch = synth.make_batch(wl, seed=8)
+    assert float(batch.advantages.abs().max()) == 0.0
+    gp, op = both_params(batch)
+    out, dH, dW = gpu_fwd_bwd(batch, gp)
+    assert float(out.loss.cpu()[0]) == 0.0 and out.stats_host()["n_active"] == 0
+    assert float(dW.abs().max()) == 0.0
+
+
+def test_target_in_last_vocabulary_column_and_tail_tile():
+    wl = synth.WORKLOADS["small"].scaled(T=200, S=2, H=128, V=1187, lengths="tiny")
+    batch = synth.make_batch(wl, seed=10)
+    batch.targets[::3] = 1186
+    batch.targets[1::3] = 1024
+    gp, op = both_params(batch)
+    check_against_oracle(batch, gp, op)
+
+
+def test_dw_accumulate_and_panel_additivity():
+    wl = synth.WORKLOADS["small"].scaled(T=600, S=3, H=128, V=1500, lengths="tiny")
+    batch = synth.make_batch(wl, seed=14)
+    gp1, _ = both_params(batch, bwd_panel_tokens=128)
+    gp2, _ = both_params(batch, bwd_panel_tokens=1024)
+    _, dH1, dW1 = gpu_fwd_bwd(batch, gp1)
+    _, dH2, dW2 = gpu_fwd_bwd(batch, gp2)
+    assert torch.equal(dH1, dH2)
+    assert rel_l2(dW1.cpu().numpy(), dW2.cpu().numpy()) <= 1e-5
+    gp3, _ = both_params(batch, dw_accumulate=True)
+    b = batch.to(DEV)
+    out = B.token_loss_fwd(gp3, b.hidden, b.W, b.targets, b.old_logp, b.segment_version, b.advantages, b.seq_offsets)
+    dW = torch.ones(wl.V, wl.H, dtype=torch.float32, device=DEV)
+    B.token_loss_bwd(gp3, b.hidden, b.W, b.targets, out.lse, out.grad_coef, d_W=dW)
+    assert rel_l2((dW - 1.0).cpu().numpy(), dW2.cpu().numpy()) <= 1e-4
+
+
+def test_empty_batch_and_bad_arguments():
+    p = B.Params(T=0, H=64, V=128, num_seqs=0, dtype="bf16")
+    ws = torch.empty(B.workspace_bytes(p), dtype=torch.uint8, device=DEV)
+    e = lambda n, dt=torch.float32: torch.zeros(n, dtype=dt, device=DEV)
+    out = B.token_loss_fwd(p, e(0, torch.bfloat16).reshape(0, 64), e(128 * 64, torch.bfloat16), e(0, torch.int32),
+                           e(0), e(0, torch.int32), e(0), e(1, torch.int32), workspace=ws)
+    torch.cuda.synchronize()
+    assert float(out.loss.cpu()[0]) == 0.0
+    bad = B.Params(T=8, H=60, V=128, num_seqs=1, dtype="bf16")           # H not a multiple of 8
+    with pytest.raises(B.UlorlError):
+        B.workspace_bytes(bad)
+    ok = B.Params(T=8, H=64, V=128, num_seqs=1, dtype="bf16")
+    small_ws = torch.empty(16, dtype=torch.uint8, device=DEV)
+    with pytest.raises(B.UlorlError, match="workspace"):
+        B.token_loss_fwd(ok, e(8 * 64, torch.bfloat16), e(128 * 64, torch.bfloat16), e(8, torch.int32), e(8),
+                         e(8, torch.int32), e(1), torch.tensor([0, 8], dtype=torch.int32, device=DEV),
+                         workspace=small_ws)
+
+
+def test_out_of_range_target_is_clamped_and_reported():
+    wl = synth.WORKLOADS["small"].scaled(T=130, S=1, H=64, V=300, lengths="single")
+    batch = synth.make_batch(wl, seed=16)
+    batch.targets[5] = 300
+    batch.targets[77] = -4
+    for path in ("tensor", "simt"):
+        gp, _ = both_params(batch, kernel_path=path)
+        b = batch.to(DEV)
+        ws = B.alloc_workspace(gp, DEV)
+        out = B.token_loss_fwd(gp, b.hidden, b.W, b.targets, b.old_logp, b.segment_version, b.advantages,
+                               b.seq_offsets, workspace=ws)
+        assert B.check_status(ws) == -6
+        assert torch.isfinite(out.logp).all()
+
+
+def test_repeated_runs_are_bit_identical():
+    wl = synth.WORKLOADS["small"].scaled(T=900, S=4, H=256, V=4000, lengths="tiny")
+    batch = synth.make_batch(wl, seed=18)
+    gp, _ = both_params(batch)
+    a = gpu_fwd_bwd(batch, gp)
+    b = gpu_fwd_bwd(batch, gp)
+    assert torch.equal(a[0].logp, b[0].logp) and torch.equal(a[0].loss, b[0].loss)
+    assert torch.equal(a[1], b[1]) and torch.equal(a[2], b[2])

@@ -1,0 +1,70 @@
+"""Host-side checks that need no GPU: the shared library loads, exports every function that
+include/ulorl.h declares, and its pure host functions behave."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2507_19766_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2507_19766_b200 import build
+    build.build()
+    return B.load_library()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "ulorl.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ulorl_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_functions()
+    assert "ulorl_token_loss_fwd" in names and "ulorl_token_loss_bwd" in names
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(B.EXPORTS) <= set(names)
+
+
+def test_struct_sizes_match_header(lib):
+    # 9 int32 + 5 float + (pad) int64 + 4 int32
+    assert ctypes.sizeof(B.CParams) == 80
+    assert ctypes.sizeof(B.CStats) == 4 * (2 + 6 + 3 * 16 + 4)
+
+
+def test_workspace_bytes_is_a_pure_host_function(lib):
+    p = B.Params(T=131072, H=2048, V=151936, num_seqs=1, dtype="bf16")
+    n = B.workspace_bytes(p)
+    # one 16384-token panel of bf16 dz dominates
+    assert 16384 * 151936 * 2 <= n <= 16384 * 151936 * 2 + (64 << 20)
+    small = B.Params(T=512, H=256, V=4096, num_seqs=4, dtype="f32")
+    assert 512 * 4096 * 4 <= B.workspace_bytes(small) <= 512 * 4096 * 4 + (4 << 20)
+    with pytest.raises(B.UlorlError):
+        B.workspace_bytes(B.Params(T=8, H=60, V=128, num_seqs=1))
+    with pytest.raises(B.UlorlError):
+        B.workspace_bytes(B.Params(T=8, H=64, V=128, num_seqs=1, inv_temperature=0.0))
+    with pytest.raises(B.UlorlError):
+        B.workspace_bytes(B.Params(T=8, H=64, V=128, num_seqs=1, dtype="f32", kernel_path="tensor"))
+
+
+def test_status_strings(lib):
+    assert B.status_string(0) == "ok"
+    assert "workspace" in B.status_string(-3)
+    assert "target" in B.status_string(-6)
+    assert B.launch_count() >= 0
+
+
+def test_null_arguments_are_rejected_without_a_device(lib):
+    p = B.Params(T=8, H=64, V=128, num_seqs=1).to_c()
+    args = [None] * 16
+    code = lib.ulorl_token_loss_fwd(ctypes.byref(p), *args, None, 0, None)
+    assert code == -1
+    code = lib.ulorl_token_loss_bwd(ctypes.byref(p), *([None] * 8), None, 0, None)
+    assert code == -1
+    assert lib.ulorl_token_loss_fwd(None, *args, None, 0, None) == -1
