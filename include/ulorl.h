@@ -147,6 +147,35 @@ const char* ulorl_status_string(int status);
 /* Number of kernel launches issued by this library since it was loaded (host counter). */
 int64_t ulorl_launch_count(void);
 
+/*
+ * Per-kernel timing of the four tensor-core kernels (0 online-softmax statistics, 1 dz recompute,
+ * 2 d_hidden, 3 d_W).  Between begin and end every such launch is bracketed by a CUDA event pair
+ * on its stream; end waits for those events and returns, per kernel, the summed duration in
+ * milliseconds (total_ms[4], host) and the number of launches (launches[4], host).  The events are
+ * created on first use and kept; this is a measurement aid, not part of the update path.
+ */
+int ulorl_kernel_timing_begin(void);
+int ulorl_kernel_timing_end(float* total_ms, int64_t* launches);
+
+/*
+ * One whole step (forward then backward of Eq. 10's objective) for a caller whose buffers live in
+ * HOST memory (pinned memory makes the copies asynchronous).  Inputs h_* are copied to the device
+ * arena, both passes run there, and every non-NULL output is copied back: h_logp[T], h_entropy[T],
+ * h_flags[T], h_seq_entropy[S], h_loss[1], h_stats (ulorl_stats_t), h_d_hidden[T,H] (params->dtype),
+ * h_d_W[V,H] (f32).  d_arena is DEVICE memory of at least ulorl_host_step_arena_bytes(params)
+ * bytes, owned by the caller and reusable across calls; it holds the device copies, the outputs
+ * and the workspace.  Asynchronous on cuda_stream: synchronise the stream before reading outputs.
+ */
+size_t ulorl_host_step_arena_bytes(const ulorl_params_t* params);
+int ulorl_token_loss_step_host(const ulorl_params_t* params,
+                               const void* h_hidden, const void* h_W, const int32_t* h_targets,
+                               const float* h_old_logp, const int32_t* h_segment_version,
+                               const float* h_advantages, const int32_t* h_seq_offsets,
+                               const float* h_entropy_supplied,
+                               float* h_logp, float* h_entropy, uint8_t* h_flags, float* h_seq_entropy,
+                               float* h_loss, void* h_stats, void* h_d_hidden, float* h_d_W,
+                               void* d_arena, size_t arena_bytes, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

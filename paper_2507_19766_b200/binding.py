@@ -59,7 +59,9 @@ class CStats(ctypes.Structure):
 
 
 EXPORTS = ("ulorl_workspace_bytes", "ulorl_token_loss_fwd", "ulorl_token_loss_decide", "ulorl_token_loss_bwd",
-           "ulorl_check_status", "ulorl_status_string", "ulorl_launch_count")
+           "ulorl_check_status", "ulorl_status_string", "ulorl_launch_count", "ulorl_kernel_timing_begin",
+           "ulorl_kernel_timing_end", "ulorl_host_step_arena_bytes", "ulorl_token_loss_step_host")
+KERNEL_KINDS = ("stats", "dz", "d_hidden", "d_W")
 
 _lib = None
 
@@ -88,6 +90,14 @@ def load_library() -> ctypes.CDLL:
     lib.ulorl_status_string.argtypes = [ctypes.c_int]
     lib.ulorl_launch_count.restype = ctypes.c_int64
     lib.ulorl_launch_count.argtypes = []
+    lib.ulorl_kernel_timing_begin.restype = ctypes.c_int
+    lib.ulorl_kernel_timing_begin.argtypes = []
+    lib.ulorl_kernel_timing_end.restype = ctypes.c_int
+    lib.ulorl_kernel_timing_end.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int64)]
+    lib.ulorl_host_step_arena_bytes.restype = ctypes.c_size_t
+    lib.ulorl_host_step_arena_bytes.argtypes = [cp]
+    lib.ulorl_token_loss_step_host.restype = ctypes.c_int
+    lib.ulorl_token_loss_step_host.argtypes = [cp] + [vp] * 16 + [vp, ctypes.c_size_t, vp]
     _lib = lib
     return lib
 
@@ -262,3 +272,43 @@ def token_loss_bwd(p: Params, hidden, W, targets, lse, grad_coef, grad_loss=None
 
 def check_status(workspace: torch.Tensor) -> int:
     return int(load_library().ulorl_check_status(_ptr(workspace), _stream()))
+
+
+def kernel_timing_begin():
+    _check(load_library().ulorl_kernel_timing_begin(), "ulorl_kernel_timing_begin")
+
+
+def kernel_timing_end() -> dict:
+    """Per tensor-core kernel: (total milliseconds, launches) since kernel_timing_begin()."""
+    ms = (ctypes.c_float * 4)()
+    n = (ctypes.c_int64 * 4)()
+    _check(load_library().ulorl_kernel_timing_end(ms, n), "ulorl_kernel_timing_end")
+    return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(KERNEL_KINDS)}
+
+
+def host_step_arena_bytes(p: Params) -> int:
+    n = load_library().ulorl_host_step_arena_bytes(ctypes.byref(p.to_c()))
+    if n == 0:
+        raise UlorlError("ulorl_host_step_arena_bytes: invalid parameters")
+    return int(n)
+
+
+def _hptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if t.is_cuda or not t.is_contiguous():
+        raise UlorlError("host-step tensors must be contiguous CPU tensors")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def token_loss_step_host(p: Params, arena: torch.Tensor, hidden, W, targets, old_logp, segment_version, advantages,
+                         seq_offsets, entropy_supplied=None, logp=None, entropy=None, flags=None, seq_entropy=None,
+                         loss=None, stats=None, d_hidden=None, d_W=None):
+    """ulorl_token_loss_step_host: every tensor except `arena` lives in host memory (pinned for
+    asynchronous copies).  Asynchronous on the current stream."""
+    code = load_library().ulorl_token_loss_step_host(
+        ctypes.byref(p.to_c()), _hptr(hidden), _hptr(W), _hptr(targets), _hptr(old_logp), _hptr(segment_version),
+        _hptr(advantages), _hptr(seq_offsets), _hptr(entropy_supplied), _hptr(logp), _hptr(entropy), _hptr(flags),
+        _hptr(seq_entropy), _hptr(loss), _hptr(stats), _hptr(d_hidden), _hptr(d_W), _ptr(arena), arena.numel(),
+        _stream())
+    _check(code, "ulorl_token_loss_step_host")

@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <vector>
 
 #include "common.cuh"
 #include "elementwise.cuh"
@@ -139,6 +140,25 @@ static int make_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uint
   return ULORL_OK;
 }
 
+// Optional per-kernel timing of the tensor-core launches: when enabled, an event pair brackets
+// every launch on its stream, so durations are measured inside whatever region the caller times.
+struct KernelTiming {
+  bool enabled = false;
+  std::vector<cudaEvent_t> ev[4];   // start/stop pairs per kernel kind
+  size_t used[4] = {0, 0, 0, 0};
+};
+static KernelTiming g_timing;
+
+static cudaEvent_t timing_event(int kind) {
+  KernelTiming& t = g_timing;
+  if (t.used[kind] == t.ev[kind].size()) {
+    cudaEvent_t e;
+    if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+    t.ev[kind].push_back(e);
+  }
+  return t.ev[kind][t.used[kind]++];
+}
+
 template <int kMode>
 static int launch_umma(const CUtensorMap& ma, const CUtensorMap& mb, const UmmaArgs& a, cudaStream_t stream) {
   static bool configured = false;
@@ -156,8 +176,16 @@ static int launch_umma(const CUtensorMap& ma, const CUtensorMap& mb, const UmmaA
   const int units = (kMode == kModeStats) ? a.m_tiles * a.n_split : a.m_tiles * a.n_tiles;
   if (units <= 0) return ULORL_OK;
   const int grid = units < num_sms ? units : num_sms;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  if (g_timing.enabled) {
+    e0 = timing_event(kMode);
+    e1 = timing_event(kMode);
+    if (e0 && e1) cudaEventRecord(e0, stream);
+  }
   umma_kernel<kMode><<<grid, kUmmaThreads, kUmmaSmemBytes, stream>>>(ma, mb, a);
-  return check_launch();
+  const int st = check_launch();
+  if (e0 && e1) cudaEventRecord(e1, stream);
+  return st;
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -467,6 +495,123 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
       ULORL_LAUNCH_CHECK();
     }
   }
+  return ULORL_OK;
+}
+
+int ulorl_kernel_timing_begin(void) {
+  for (int k = 0; k < 4; ++k) g_timing.used[k] = 0;
+  g_timing.enabled = true;
+  return ULORL_OK;
+}
+
+int ulorl_kernel_timing_end(float* total_ms, int64_t* launches) {
+  g_timing.enabled = false;
+  if (!total_ms || !launches) return ULORL_ERR_INVALID_ARG;
+  for (int k = 0; k < 4; ++k) {
+    double tot = 0.0;
+    int64_t n = 0;
+    for (size_t i = 0; i + 1 < g_timing.used[k]; i += 2) {
+      if (cudaEventSynchronize(g_timing.ev[k][i + 1]) != cudaSuccess) return ULORL_ERR_CUDA;
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, g_timing.ev[k][i], g_timing.ev[k][i + 1]) != cudaSuccess) return ULORL_ERR_CUDA;
+      tot += ms;
+      ++n;
+    }
+    total_ms[k] = (float)tot;
+    launches[k] = n;
+  }
+  return ULORL_OK;
+}
+
+// ------------------------------------------------------------------ host-buffer step
+namespace {
+struct HostStepLayout {
+  size_t hidden, W, targets, old_logp, segver, adv, seq_off, ent_sup;
+  size_t logp, entropy, lse, grad_coef, flags, seq_entropy, loss, stats, d_hidden, d_W, ws, total;
+  size_t elem;
+};
+HostStepLayout host_step_layout(const ulorl_params_t* p) {
+  HostStepLayout L{};
+  const size_t T = (size_t)p->T, H = (size_t)p->H, V = (size_t)p->V, S = (size_t)(p->num_seqs > 0 ? p->num_seqs : 1);
+  L.elem = p->dtype == ULORL_BF16 ? 2 : 4;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { const size_t o = off; off = align_up(off + (bytes ? bytes : 16), 1024); return o; };
+  L.hidden = take(T * H * L.elem);
+  L.W = take(V * H * L.elem);
+  L.targets = take(T * 4);
+  L.old_logp = take(T * 4);
+  L.segver = take(T * 4);
+  L.adv = take((p->adv_per_token ? T : S) * 4);
+  L.seq_off = take((S + 1) * 4);
+  L.ent_sup = take(S * 4);
+  L.logp = take(T * 4);
+  L.entropy = take(T * 4);
+  L.lse = take(T * 4);
+  L.grad_coef = take(T * 4);
+  L.flags = take(T);
+  L.seq_entropy = take(S * 4);
+  L.loss = take(16);
+  L.stats = take(sizeof(ulorl_stats_t));
+  L.d_hidden = take(T * H * L.elem);
+  L.d_W = take(V * H * 4);
+  L.ws = take(make_plan(p).total);
+  L.total = off;
+  return L;
+}
+}  // namespace
+
+size_t ulorl_host_step_arena_bytes(const ulorl_params_t* params) {
+  if (validate_params(params) != ULORL_OK) return 0;
+  return host_step_layout(params).total;
+}
+
+int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidden, const void* h_W,
+                               const int32_t* h_targets, const float* h_old_logp, const int32_t* h_segment_version,
+                               const float* h_advantages, const int32_t* h_seq_offsets,
+                               const float* h_entropy_supplied, float* h_logp, float* h_entropy, uint8_t* h_flags,
+                               float* h_seq_entropy, float* h_loss, void* h_stats, void* h_d_hidden, float* h_d_W,
+                               void* d_arena, size_t arena_bytes, void* cuda_stream) {
+  int st = validate_params(params);
+  if (st != ULORL_OK) return st;
+  if (!d_arena || !h_loss) return ULORL_ERR_INVALID_ARG;
+  if (params->T > 0 && (!h_hidden || !h_W || !h_targets || !h_advantages || !h_seq_offsets)) return ULORL_ERR_INVALID_ARG;
+  const HostStepLayout L = host_step_layout(params);
+  if (arena_bytes < L.total) return ULORL_ERR_WORKSPACE;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  uint8_t* a = reinterpret_cast<uint8_t*>(d_arena);
+  const size_t T = (size_t)params->T, H = (size_t)params->H, V = (size_t)params->V, S = (size_t)params->num_seqs;
+  auto h2d = [&](size_t off, const void* src, size_t bytes) {
+    return (!src || !bytes) ? cudaSuccess : cudaMemcpyAsync(a + off, src, bytes, cudaMemcpyHostToDevice, stream);
+  };
+  auto d2h = [&](void* dst, size_t off, size_t bytes) {
+    return (!dst || !bytes) ? cudaSuccess : cudaMemcpyAsync(dst, a + off, bytes, cudaMemcpyDeviceToHost, stream);
+  };
+  if (h2d(L.hidden, h_hidden, T * H * L.elem) != cudaSuccess || h2d(L.W, h_W, V * H * L.elem) != cudaSuccess ||
+      h2d(L.targets, h_targets, T * 4) != cudaSuccess || h2d(L.old_logp, h_old_logp, T * 4) != cudaSuccess ||
+      h2d(L.segver, h_segment_version, T * 4) != cudaSuccess ||
+      h2d(L.adv, h_advantages, (params->adv_per_token ? T : S) * 4) != cudaSuccess ||
+      h2d(L.seq_off, h_seq_offsets, (S + 1) * 4) != cudaSuccess || h2d(L.ent_sup, h_entropy_supplied, S * 4) != cudaSuccess)
+    return ULORL_ERR_CUDA;
+  st = ulorl_token_loss_fwd(params, a + L.hidden, a + L.W, reinterpret_cast<const int32_t*>(a + L.targets),
+                            h_old_logp ? reinterpret_cast<const float*>(a + L.old_logp) : nullptr,
+                            h_segment_version ? reinterpret_cast<const int32_t*>(a + L.segver) : nullptr,
+                            reinterpret_cast<const float*>(a + L.adv), reinterpret_cast<const int32_t*>(a + L.seq_off),
+                            h_entropy_supplied ? reinterpret_cast<const float*>(a + L.ent_sup) : nullptr,
+                            reinterpret_cast<float*>(a + L.logp), reinterpret_cast<float*>(a + L.entropy),
+                            reinterpret_cast<float*>(a + L.lse), reinterpret_cast<float*>(a + L.grad_coef), a + L.flags,
+                            reinterpret_cast<float*>(a + L.seq_entropy), reinterpret_cast<float*>(a + L.loss),
+                            a + L.stats, a + L.ws, L.total - L.ws, stream);
+  if (st != ULORL_OK) return st;
+  st = ulorl_token_loss_bwd(params, a + L.hidden, a + L.W, reinterpret_cast<const int32_t*>(a + L.targets),
+                            reinterpret_cast<const float*>(a + L.lse), reinterpret_cast<const float*>(a + L.grad_coef),
+                            nullptr, a + L.d_hidden, reinterpret_cast<float*>(a + L.d_W), a + L.ws, L.total - L.ws,
+                            stream);
+  if (st != ULORL_OK) return st;
+  if (d2h(h_logp, L.logp, T * 4) != cudaSuccess || d2h(h_entropy, L.entropy, T * 4) != cudaSuccess ||
+      d2h(h_flags, L.flags, T) != cudaSuccess || d2h(h_seq_entropy, L.seq_entropy, S * 4) != cudaSuccess ||
+      d2h(h_loss, L.loss, 4) != cudaSuccess || d2h(h_stats, L.stats, sizeof(ulorl_stats_t)) != cudaSuccess ||
+      d2h(h_d_hidden, L.d_hidden, T * H * L.elem) != cudaSuccess || d2h(h_d_W, L.d_W, V * H * 4) != cudaSuccess)
+    return ULORL_ERR_CUDA;
   return ULORL_OK;
 }
 

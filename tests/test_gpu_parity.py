@@ -77,9 +77,13 @@ def check_against_oracle(batch, gp, op, grad_loss=None, check_grads=True):
         eh = rel_l2(dH.float().cpu().numpy(), dH_ref)
         ew = rel_l2(dW.cpu().numpy(), dW_ref)
         assert eh <= TOL_GRAD and ew <= TOL_GRAD, (eh, ew)
-        # sum_v dz[t, v] = 0, so the column sums of d_W vanish
+        # sum_v dz[t, v] = 0, so the column sums of d_W vanish up to the rounding of dz: the tensor path
+        # stores dz in bf16 (relative error 2^-9 per element, sum_v |dz[t, v]| <= 2 |coef_t|), so
+        # |colsum_h| <= 2^-8 sum_t |coef_t| |hidden[t, h]|; the float32 path is held to 1e-5 of that sum
         col = np.abs(dW.double().sum(dim=0).cpu().numpy()).max()
-        assert col <= 1e-3 * max(1e-12, float(dW.abs().max()))
+        coef_sum = float(np.abs(g).sum()) * op.inv_temperature * (1.0 if grad_loss is None else abs(grad_loss))
+        unit = 2.0 ** -8 if (gp.dtype == "bf16" and gp.kernel_path != "simt") else 1e-5
+        assert col <= unit * coef_sum * float(np.abs(oi["hidden"]).max()) + 1e-12
     return out, ref
 
 
