@@ -39,7 +39,8 @@ typedef enum {
   ULORL_ERR_WORKSPACE = -3,     /* workspace smaller than ulorl_workspace_bytes()       */
   ULORL_ERR_CUDA = -4,          /* a CUDA runtime or driver call failed                 */
   ULORL_ERR_DEVICE_TIMEOUT = -5,/* a bounded device-side wait ran out                   */
-  ULORL_ERR_BAD_TARGET = -6     /* some target id was outside [0, V) (row was clamped)  */
+  ULORL_ERR_BAD_TARGET = -6,    /* some target id was outside [0, V) (row was clamped)  */
+  ULORL_ERR_STATIC_LIMIT = -7   /* batch exceeds the built-in scratch of ulorl_token_loss_decide_static */
 } ulorl_status_t;
 
 typedef enum { ULORL_F32 = 0, ULORL_BF16 = 1 } ulorl_dtype_t;
@@ -124,6 +125,39 @@ int ulorl_token_loss_decide(const ulorl_params_t* params,
                             const float* entropy_supplied,
                             float* grad_coef, uint8_t* flags, float* seq_entropy, float* loss,
                             void* stats, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * The same elementwise stage as ulorl_token_loss_decide for callers that cannot hand over a
+ * workspace because they cannot allocate device memory at the point of the call: code running
+ * inside another framework's step where the allocator is frozen (a memory plan fixed ahead of
+ * time, a pool that is full by design), plugins that only receive the tensors of the op they
+ * implement, or a process whose memory budget was handed out entirely at start-up.  (The paper
+ * has no counterpart to this function; it is a packaging variant, not a step of the method.)
+ *
+ * The scratch that ulorl_token_loss_decide takes from the caller's workspace (status word,
+ * per-sequence float64 entropy sums, one partial record per 256 tokens) lives instead in a fixed
+ * array inside the library's device image: about 1.7 MB on every GPU that loads the library,
+ * held until the process exits.  Limits: T <= ULORL_STATIC_MAX_TOKENS and num_seqs <=
+ * ULORL_STATIC_MAX_SEQS; larger batches are rejected with ULORL_ERR_STATIC_LIMIT (and a message
+ * on stderr) before anything is launched.  Inputs and outputs are the caller's device buffers,
+ * exactly as for ulorl_token_loss_decide; results are identical.
+ *
+ * The function calls no allocating routine.  Its first call on a device looks up the device
+ * address of the array (one runtime query with that device current) and keeps it; make that
+ * first call outside any stream capture.  All calls on a device share the one array, which keeps
+ * the previous call's contents (the call clears the status word itself): two calls whose kernels
+ * can overlap on the GPU -- different streams without an ordering between them -- race on it and
+ * give wrong results.  Calls on one stream are ordered and safe.
+ */
+#define ULORL_STATIC_MAX_TOKENS (1 << 20)
+#define ULORL_STATIC_MAX_SEQS   (1 << 16)
+int ulorl_token_loss_decide_static(const ulorl_params_t* params,
+                                   const float* logp, const float* entropy,
+                                   const float* old_logp, const int32_t* segment_version,
+                                   const float* advantages, const int32_t* seq_offsets,
+                                   const float* entropy_supplied,
+                                   float* grad_coef, uint8_t* flags, float* seq_entropy, float* loss,
+                                   void* stats, void* cuda_stream);
 
 /*
  * Backward (chain rule through Eq. 6): with dz[t,v] = kappa * grad_loss * grad_coef[t] *

@@ -60,7 +60,9 @@ class CStats(ctypes.Structure):
 
 EXPORTS = ("ulorl_workspace_bytes", "ulorl_token_loss_fwd", "ulorl_token_loss_decide", "ulorl_token_loss_bwd",
            "ulorl_check_status", "ulorl_status_string", "ulorl_launch_count", "ulorl_kernel_timing_begin",
-           "ulorl_kernel_timing_end", "ulorl_host_step_arena_bytes", "ulorl_token_loss_step_host")
+           "ulorl_kernel_timing_end", "ulorl_host_step_arena_bytes", "ulorl_token_loss_step_host",
+           "ulorl_token_loss_decide_static")
+STATIC_MAX_TOKENS, STATIC_MAX_SEQS = 1 << 20, 1 << 16
 KERNEL_KINDS = ("stats", "dz", "d_hidden", "d_W")
 
 _lib = None
@@ -82,6 +84,8 @@ def load_library() -> ctypes.CDLL:
     lib.ulorl_token_loss_fwd.argtypes = [cp] + [vp] * 16 + [vp, ctypes.c_size_t, vp]
     lib.ulorl_token_loss_decide.restype = ctypes.c_int
     lib.ulorl_token_loss_decide.argtypes = [cp] + [vp] * 12 + [vp, ctypes.c_size_t, vp]
+    lib.ulorl_token_loss_decide_static.restype = ctypes.c_int
+    lib.ulorl_token_loss_decide_static.argtypes = [cp] + [vp] * 12 + [vp]
     lib.ulorl_token_loss_bwd.restype = ctypes.c_int
     lib.ulorl_token_loss_bwd.argtypes = [cp] + [vp] * 8 + [vp, ctypes.c_size_t, vp]
     lib.ulorl_check_status.restype = ctypes.c_int
@@ -248,6 +252,25 @@ def token_loss_decide(p: Params, logp, entropy, old_logp, segment_version, advan
         _ptr(seq_offsets), _ptr(entropy_supplied), _ptr(out.grad_coef), _ptr(out.flags), _ptr(out.seq_entropy),
         _ptr(out.loss), _ptr(out.stats), _ptr(workspace), workspace.numel(), _stream())
     _check(code, "ulorl_token_loss_decide")
+    return out
+
+
+def token_loss_decide_static(p: Params, logp, entropy, old_logp, segment_version, advantages, seq_offsets,
+                             entropy_supplied=None, out: Optional[FwdOut] = None) -> FwdOut:
+    """ulorl_token_loss_decide_static: the elementwise stage with no workspace argument, for callers
+    that cannot allocate device memory; its scratch is a fixed array inside the library (at most
+    STATIC_MAX_TOKENS tokens and STATIC_MAX_SEQS sequences).  `out` must be given by such a caller;
+    when omitted this wrapper allocates the outputs with torch for convenience."""
+    lib = load_library()
+    _want(logp, torch.float32, p.T, "logp")
+    _want(entropy, torch.float32, p.T, "entropy")
+    out = out or alloc_fwd_outputs(p, logp.device)
+    out.logp, out.entropy = logp, entropy
+    code = lib.ulorl_token_loss_decide_static(
+        ctypes.byref(p.to_c()), _ptr(logp), _ptr(entropy), _ptr(old_logp), _ptr(segment_version), _ptr(advantages),
+        _ptr(seq_offsets), _ptr(entropy_supplied), _ptr(out.grad_coef), _ptr(out.flags), _ptr(out.seq_entropy),
+        _ptr(out.loss), _ptr(out.stats), _stream())
+    _check(code, "ulorl_token_loss_decide_static")
     return out
 
 

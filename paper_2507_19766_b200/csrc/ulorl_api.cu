@@ -278,6 +278,7 @@ const char* ulorl_status_string(int status) {
     case ULORL_ERR_CUDA: return "CUDA call failed";
     case ULORL_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
     case ULORL_ERR_BAD_TARGET: return "a target id was outside [0, V)";
+    case ULORL_ERR_STATIC_LIMIT: return "batch larger than the built-in scratch of the no-allocation entry point";
     default: return "unknown status";
   }
 }
@@ -496,6 +497,73 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
     }
   }
   return ULORL_OK;
+}
+
+// ------------------------------------------------------------------ decision stage without a workspace
+// Scratch of ulorl_token_loss_decide_static: a fixed array in the library's own device image,
+// resident on every GPU that loads the library until the process exits.
+//   [0, 256)                       status word and batch-mean slot
+//   [256, 256 + 8 * max seqs)      float64 entropy sum per sequence
+//   rest                           one DecidePartial per block of 256 tokens
+constexpr size_t kStaticSeqBytes = sizeof(double) * (size_t)ULORL_STATIC_MAX_SEQS;
+constexpr size_t kStaticDecideBlocks = ((size_t)ULORL_STATIC_MAX_TOKENS + kDecideThreads - 1) / kDecideThreads;
+constexpr size_t kStaticScratchBytes = 256 + kStaticSeqBytes + sizeof(DecidePartial) * kStaticDecideBlocks;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// Device address of g_static_scratch on the current device.  In host code the array's name is only
+// a handle for the runtime; the address a kernel can use comes from cudaGetSymbolAddress, asked once
+// per device with that device current.
+static int static_scratch_address(uint8_t** out) {
+  constexpr int kMaxDevices = 64;
+  static uint8_t* cached[kMaxDevices] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ULORL_ERR_CUDA;
+  if (!cached[dev]) {
+    void* ptr = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (e != cudaSuccess || !ptr) {
+      std::fprintf(stderr, "ulorl: cudaGetSymbolAddress failed: %s\n", cudaGetErrorString(e));
+      return ULORL_ERR_CUDA;
+    }
+    cached[dev] = static_cast<uint8_t*>(ptr);
+  }
+  *out = cached[dev];
+  return ULORL_OK;
+}
+
+int ulorl_token_loss_decide_static(const ulorl_params_t* params, const float* logp, const float* entropy,
+                                   const float* old_logp, const int32_t* segment_version, const float* advantages,
+                                   const int32_t* seq_offsets, const float* entropy_supplied, float* grad_coef,
+                                   uint8_t* flags, float* seq_entropy, float* loss, void* stats, void* cuda_stream) {
+  int st = validate_params(params);
+  if (st != ULORL_OK) return st;
+  if (params->T > ULORL_STATIC_MAX_TOKENS || params->num_seqs > ULORL_STATIC_MAX_SEQS) {
+    std::fprintf(stderr,
+                 "ulorl_token_loss_decide_static: T=%d, num_seqs=%d exceed the built-in scratch (at most %d tokens, "
+                 "%d sequences); use ulorl_token_loss_decide with a caller workspace\n",
+                 params->T, params->num_seqs, ULORL_STATIC_MAX_TOKENS, ULORL_STATIC_MAX_SEQS);
+    return ULORL_ERR_STATIC_LIMIT;
+  }
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  uint8_t* ws = nullptr;
+  st = static_scratch_address(&ws);
+  if (st != ULORL_OK) return st;
+  if (params->T == 0) return empty_forward(ws, 256, loss, stats, stream);
+  if (!logp || !entropy) return ULORL_ERR_INVALID_ARG;
+  st = validate_decide_args(params, old_logp, advantages, seq_offsets, entropy_supplied, seq_entropy, loss);
+  if (st != ULORL_OK) return st;
+  Plan pl{};
+  pl.off_status = 0;
+  pl.off_batch_mean = 16;
+  pl.off_seq_sum = 256;
+  pl.off_decide = 256 + kStaticSeqBytes;
+  pl.decide_blocks = (params->T + kDecideThreads - 1) / kDecideThreads;
+  pl.total = kStaticScratchBytes;
+  // the array keeps whatever the previous call left: the status word must start at zero, every
+  // other slot that this call reads is written by this call first
+  if (cudaMemsetAsync(ws + pl.off_status, 0, 256, stream) != cudaSuccess) return ULORL_ERR_CUDA;
+  return run_decide(params, pl, logp, entropy, old_logp, segment_version, advantages, seq_offsets, entropy_supplied,
+                    grad_coef, flags, seq_entropy, loss, stats, ws, stream);
 }
 
 int ulorl_kernel_timing_begin(void) {
