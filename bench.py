@@ -184,6 +184,9 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=768, help="rows of the CPU-baseline sample (0 = skip)")
     ap.add_argument("--ref-rows", type=int, default=256)
     ap.add_argument("--panel", type=int, default=0, help="backward panel tokens (0 = library default)")
+    ap.add_argument("--tokens", type=int, default=0,
+                    help="run the workload's recipe at this many tokens instead of its own T (small cases for "
+                         "profiler captures; not the benchmark configuration)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -202,7 +205,9 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     wl = synth.WORKLOADS[args.workload]
-    warmup = max(args.warmup, 3)
+    if args.tokens > 0:
+        wl = wl.scaled(T=args.tokens, S=1, lengths="single", segment_len=max(1, args.tokens // wl.max_segments))
+    warmup = max(args.warmup, 3) if args.tokens == 0 else args.warmup
     host_batch = synth.make_batch(wl, seed=synth.BASE_SEED + wl.index + 1000 * rank, device=str(dev))
     b = host_batch.to(dev)
     gp = B.Params(T=wl.T, H=wl.H, V=wl.V, num_seqs=wl.S, dtype=wl.dtype, is_mode=wl.is_mode, mpt_mode=wl.mpt_mode,
@@ -313,7 +318,7 @@ def main():
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": wl.dtype, "data": "synthetic",
-        "config": {"workload": wl.name, "T": wl.T, "H": wl.H, "V": wl.V, "sequences": wl.S,
+        "config": {"workload": wl.name + (" (reduced T)" if args.tokens > 0 else ""), "T": wl.T, "H": wl.H, "V": wl.V, "sequences": wl.S,
                    "is_mode": wl.is_mode, "mpt_mode": wl.mpt_mode, "l2": "inputs larger than L2 (hidden + W = 1.1 GB)",
                    "parallelism": f"dp{world}"},
         "tensor_frac": {"executed_tflops_per_gpu": exec_tflops / world,

@@ -9,8 +9,8 @@ namespace ulorl {
 // ------------------------------------------------------------------------------------------
 // Merge of the online-softmax partials of the vocabulary splits (log-softmax of Eq. 6, entropy
 // of Eq. 10).  partials[split][t] = (m, s, u, -) with m the running max of the raw accumulator
-// a = hidden . W[v], s = sum_v exp(kappa (a_v - m)), u = sum_v exp(kappa (a_v - m)) a_v.
-//   lse = kappa m* + ln s*,  logp = kappa a_y - lse,  Hent = lse - kappa u* / s*.
+// a = hidden . W[v], s = sum_v exp(kappa (a_v - m)), u = sum_v exp(kappa (a_v - m)) (a_v - m).
+//   lse = kappa m* + ln s*,  logp = kappa a_y - lse,  Hent = ln s* - kappa u* / s*.
 // ------------------------------------------------------------------------------------------
 __global__ void merge_splits_kernel(int T, int n_split, float kappa, const float4* __restrict__ partials,
                                     const float* __restrict__ acc_y, float* __restrict__ logp,
@@ -22,15 +22,17 @@ __global__ void merge_splits_kernel(int T, int n_split, float kappa, const float
   float s = 0.f, u = 0.f;
   for (int k = 0; k < n_split; ++k) {
     const float4 p = partials[(size_t)k * T + t];
-    if (p.x == -INFINITY) continue;
-    const float w = __expf(kappa * (p.x - m));
+    if (!(p.y > 0.f)) continue;
+    const float d = p.x - m;
+    const float w = expf(kappa * d);
     s = fmaf(p.y, w, s);
-    u = fmaf(p.z, w, u);
+    u = fmaf(w, fmaf(d, p.y, p.z), u);
   }
-  const float l = fmaf(kappa, m, logf(s));
+  const float ln_s = logf(s);
+  const float l = fmaf(kappa, m, ln_s);
   if (lse) lse[t] = l;
   if (logp) logp[t] = fmaf(kappa, acc_y[t], -l);
-  if (entropy) entropy[t] = fmaxf(l - kappa * u / s, 0.f);
+  if (entropy) entropy[t] = fmaxf(ln_s - kappa * u / s, 0.f);
 }
 
 // ------------------------------------------------------------------------------------------

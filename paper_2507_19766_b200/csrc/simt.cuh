@@ -54,7 +54,7 @@ __device__ __forceinline__ void simt_logits_tile(const TIn* __restrict__ hidden,
 }
 
 // Forward statistics.  grid = (token tiles, vocabulary splits).  Each thread keeps running
-// (max, sum exp, sum exp*a) for its four rows over the columns it owns; the sixteen threads that
+// (max m, sum exp(kappa (a - m)), sum exp(kappa (a - m)) (a - m)) for its four rows over the columns it owns; the sixteen threads that
 // share a row are merged with warp shuffles once at the end.
 template <typename TIn>
 __global__ void __launch_bounds__(kSimtThreads)
@@ -98,20 +98,27 @@ simt_stats_kernel(const TIn* __restrict__ hidden, const TIn* __restrict__ W, con
       }
       if (cmax == -INFINITY) continue;
       const float mn = fmaxf(m[i], cmax);
-      const float sc = expf(kappa * (m[i] - mn));
-      s[i] *= sc;
-      u[i] *= sc;
+      if (s[i] > 0.f) {                               // move the running sums to the new max
+        const float d = m[i] - mn;
+        const float sc = expf(kappa * d);
+        u[i] = sc * fmaf(d, s[i], u[i]);
+        s[i] *= sc;
+      }
       m[i] = mn;
+      float ls = 0.f, lu = 0.f;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int col = col0 + tx * 4 + j;
         if (col < V) {
-          const float e = expf(kappa * (acc[i][j] - mn));
-          s[i] += e;
-          u[i] = fmaf(e, acc[i][j], u[i]);
+          const float t = acc[i][j] - mn;
+          const float e = expf(kappa * t);
+          ls += e;
+          lu = fmaf(e, t, lu);
           if (col == y[i] && row0 + ty * 4 + i < T) acc_y[row0 + ty * 4 + i] = acc[i][j];
         }
       }
+      s[i] += ls;
+      u[i] += lu;
     }
   }
   // merge the sixteen column owners of each row (lanes differing in the low four bits)
@@ -124,9 +131,19 @@ simt_stats_kernel(const TIn* __restrict__ hidden, const TIn* __restrict__ W, con
       const float uo = __shfl_xor_sync(0xffffffffu, u[i], off);
       const float mn = fmaxf(m[i], mo);
       if (mn != -INFINITY) {
-        const float wa = expf(kappa * (m[i] - mn)), wb = expf(kappa * (mo - mn));
-        s[i] = s[i] * wa + so * wb;
-        u[i] = u[i] * wa + uo * wb;
+        float sa = 0.f, ua = 0.f, sb = 0.f, ub = 0.f;
+        if (s[i] > 0.f) {
+          const float d = m[i] - mn, w = expf(kappa * d);
+          sa = s[i] * w;
+          ua = w * fmaf(d, s[i], u[i]);
+        }
+        if (so > 0.f) {
+          const float d = mo - mn, w = expf(kappa * d);
+          sb = so * w;
+          ub = w * fmaf(d, so, uo);
+        }
+        s[i] = sa + sb;
+        u[i] = ua + ub;
         m[i] = mn;
       }
     }

@@ -18,6 +18,7 @@ static std::atomic<long long> g_launches{0};
 constexpr int kDesignSMs = 148;           // the plan (splits, workspace) is sized for a B200
 constexpr int kDefaultPanelTensor = 16384;
 constexpr int kDefaultPanelSimt = 1024;
+constexpr int kRasterGroup = 16;          // row tiles per raster group of the tensor-core kernels
 
 struct Plan {
   bool tensor;            // tensor-core path (bf16) or SIMT path
@@ -175,6 +176,7 @@ static int launch_umma(const CUtensorMap& ma, const CUtensorMap& mb, const UmmaA
   }
   const int units = (kMode == kModeStats) ? a.m_tiles * a.n_split : a.m_tiles * a.n_tiles;
   if (units <= 0) return ULORL_OK;
+  if (kMode != kModeStats && a.group_m <= 0) return ULORL_ERR_INVALID_ARG;
   const int grid = units < num_sms ? units : num_sms;
   cudaEvent_t e0 = nullptr, e1 = nullptr;
   if (g_timing.enabled) {
@@ -416,6 +418,7 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
         a.M = rows; a.N = V; a.K = H;
         a.m_tiles = (rows + kBM - 1) / kBM;
         a.n_tiles = (int)(pl.dz_ld / kBN) + ((pl.dz_ld % kBN) ? 1 : 0);
+        a.group_m = kRasterGroup;
         a.a_mn0 = t0;
         a.row0 = t0;
         a.kappa = kappa;
@@ -436,6 +439,7 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
         a.M = rows; a.N = H; a.K = V;
         a.m_tiles = (rows + kBM - 1) / kBM;
         a.n_tiles = (H + kBN - 1) / kBN;
+        a.group_m = kRasterGroup;
         a.row0 = t0;
         a.d_hidden = static_cast<__nv_bfloat16*>(d_hidden);
         a.out_ld = (size_t)H;
@@ -449,6 +453,7 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
         a.M = V; a.N = H; a.K = rows;
         a.m_tiles = (V + kBM - 1) / kBM;
         a.n_tiles = (H + kBN - 1) / kBN;
+        a.group_m = kRasterGroup;
         a.b_k0 = t0;
         a.d_W = d_W;
         a.out_ld = (size_t)H;

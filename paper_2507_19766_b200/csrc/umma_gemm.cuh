@@ -42,6 +42,7 @@ struct UmmaArgs {
   int m_tiles, n_tiles;     // ceil(M / kBM), ceil(N / kBN)
   int n_split;              // kModeStats: vocabulary splits; a unit is (token tile, split)
   int tiles_per_split;
+  int group_m;              // other modes: token tiles per raster group (tiles of a group run m-fastest)
   int a_mn0, a_k0;          // coordinate offsets of operand A in its tensor map (MN index, K index)
   int b_mn0, b_k0;
   int row0;                 // global token (or vocabulary row) index of accumulator row 0 of tile 0
@@ -69,10 +70,84 @@ struct ModeTraits {
   static constexpr bool b_mn = (kMode == kModeDHidden || kMode == kModeDW);
 };
 
+// Raster of the (m, n) output tiles for the modes without vocabulary splits: groups of `group_m`
+// row tiles, m fastest inside a group, so that the CTAs running at one time share a few B tiles and
+// keep the group's A tiles resident in L2 instead of streaming all of B once per row tile.
+__device__ __forceinline__ void unit_to_tile(int unit, const UmmaArgs& args, int& m_tile, int& n_tile) {
+  const int per_group = args.group_m * args.n_tiles;
+  const int group = unit / per_group;
+  const int first_m = group * args.group_m;
+  const int rows = min(args.group_m, args.m_tiles - first_m);
+  const int local = unit - group * per_group;
+  m_tile = first_m + local % rows;
+  n_tile = local / rows;
+}
+
 __device__ __forceinline__ float ex2f(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// One 32-column chunk of a row folded into the running (m, s, u) with m the max of the raw
+// accumulators a, s = sum 2^(c2 (a - m)) and u = sum 2^(c2 (a - m)) (a - m).  Keeping u relative to the
+// max makes the entropy ln s - kappa u / s free of cancellation for sharply peaked rows, and the
+// chunk's terms are summed among themselves before they meet the running totals, so 10^5 tiny
+// terms are not lost one by one against a total near one.
+template <bool kFull>
+__device__ __forceinline__ void stats_chunk(const uint32_t (&raw)[32], int nvalid, float c2, float& run_m,
+                                            float& run_s, float& run_u) {
+  float cmax = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < 32; ++j)
+    if (kFull || j < nvalid) cmax = fmaxf(cmax, __uint_as_float(raw[j]));
+  const float m_new = fmaxf(run_m, cmax);
+  if (run_s > 0.f) {                                  // move the running sums to the new max
+    const float d = run_m - m_new;                    // <= 0
+    const float sc = ex2f(d * c2);
+    run_u = sc * fmaf(d, run_s, run_u);
+    run_s *= sc;
+  }
+  run_m = m_new;
+  float s0 = 0.f, s1 = 0.f, u0 = 0.f, u1 = 0.f;       // two chains for instruction-level parallelism
+#pragma unroll
+  for (int j = 0; j < 32; j += 2) {
+    if (kFull || j < nvalid) {
+      const float t = __uint_as_float(raw[j]) - m_new;
+      const float e = ex2f(t * c2);
+      s0 += e;
+      u0 = fmaf(e, t, u0);
+    }
+    if (kFull || j + 1 < nvalid) {
+      const float t = __uint_as_float(raw[j + 1]) - m_new;
+      const float e = ex2f(t * c2);
+      s1 += e;
+      u1 = fmaf(e, t, u1);
+    }
+  }
+  run_s += s0 + s1;
+  run_u += u0 + u1;
+}
+
+// One 32-column chunk of dz = coef * (onehot - 2^(c2 a - lse2)), packed to bf16 pairs; columns at or
+// beyond nvalid give zero.  y_rel is the target column relative to the chunk (any value if outside).
+template <bool kFull>
+__device__ __forceinline__ void dz_chunk(const uint32_t (&raw)[32], int nvalid, int y_rel, float coef, float c2,
+                                         float lse2, uint32_t (&packed)[16]) {
+#pragma unroll
+  for (int j = 0; j < 32; j += 2) {
+    float v0 = 0.f, v1 = 0.f;
+    if (kFull || j < nvalid) {
+      const float p = ex2f(fmaf(__uint_as_float(raw[j]), c2, -lse2));
+      v0 = coef * ((j == y_rel ? 1.f : 0.f) - p);
+    }
+    if (kFull || j + 1 < nvalid) {
+      const float p = ex2f(fmaf(__uint_as_float(raw[j + 1]), c2, -lse2));
+      v1 = coef * ((j + 1 == y_rel ? 1.f : 0.f) - p);
+    }
+    __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+    packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
+  }
 }
 
 template <int kMode>
@@ -134,8 +209,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         n_begin = (unit % args.n_split) * args.tiles_per_split;
         n_end = min(args.n_tiles, n_begin + args.tiles_per_split);
       } else {
-        m_tile = unit / args.n_tiles;
-        n_begin = unit % args.n_tiles;
+        unit_to_tile(unit, args, m_tile, n_begin);
         n_end = n_begin + 1;
       }
       for (int n_tile = n_begin; n_tile < n_end; ++n_tile) {
@@ -236,8 +310,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         n_begin = split * args.tiles_per_split;
         n_end = min(args.n_tiles, n_begin + args.tiles_per_split);
       } else {
-        m_tile = unit / args.n_tiles;
-        n_begin = unit % args.n_tiles;
+        unit_to_tile(unit, args, m_tile, n_begin);
         n_end = n_begin + 1;
       }
       const int row = m_tile * kBM + row_in_tile;       // row within this launch's M extent
@@ -283,25 +356,8 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           const int nvalid = min(32, args.N - col0);           // may be <= 0 only in kModeDz padding
 
           if (kMode == kModeStats) {
-            float cmax = -INFINITY;
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (j < nvalid) cmax = fmaxf(cmax, __uint_as_float(raw[j]));
-            const float m_new = fmaxf(run_m, cmax);
-            const float sc = ex2f((run_m - m_new) * c2);        // first chunk: 2^(-inf) = 0
-            run_s *= sc;
-            run_u *= sc;
-            run_m = m_new;
-            const float off = -m_new * c2;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              if (j < nvalid) {
-                const float a = __uint_as_float(raw[j]);
-                const float e = ex2f(fmaf(a, c2, off));
-                run_s += e;
-                run_u = fmaf(e, a, run_u);
-              }
-            }
+            if (nvalid >= 32) stats_chunk<true>(raw, 32, c2, run_m, run_s, run_u);
+            else stats_chunk<false>(raw, nvalid, c2, run_m, run_s, run_u);
             if (row_ok && y >= col0 && y < col0 + 32) {
               float ay = 0.f;
 #pragma unroll
@@ -310,20 +366,8 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             }
           } else if (kMode == kModeDz) {
             uint32_t packed[16];
-#pragma unroll
-            for (int j = 0; j < 32; j += 2) {
-              float v0 = 0.f, v1 = 0.f;
-              if (j < nvalid) {
-                const float p = ex2f(fmaf(__uint_as_float(raw[j]), c2, -lse2));
-                v0 = coef * ((col0 + j == y ? 1.f : 0.f) - p);
-              }
-              if (j + 1 < nvalid) {
-                const float p = ex2f(fmaf(__uint_as_float(raw[j + 1]), c2, -lse2));
-                v1 = coef * ((col0 + j + 1 == y ? 1.f : 0.f) - p);
-              }
-              __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
-              packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
-            }
+            if (nvalid >= 32) dz_chunk<true>(raw, 32, y - col0, coef, c2, lse2, packed);
+            else dz_chunk<false>(raw, nvalid, y - col0, coef, c2, lse2, packed);
             if (row_ok) {
               uint4* dst = reinterpret_cast<uint4*>(args.dz + (size_t)row * args.dz_ld + col0);
               const int ncols = min(32, args.dz_cols - col0);     // multiple of 8

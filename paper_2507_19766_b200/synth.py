@@ -72,7 +72,12 @@ WORKLOADS = {
     "ultra": Workload("ultra", 4, T=131072, S=1, H=2048, V=151936, dtype="bf16",
                       lengths="single", segment_len=16384, max_segments=8,
                       noise="stale:0.02", adv="plus1", planted=0.7, sampled=0.3,
-                      mpt_mode="dynamic", beta_planted=(24.0, 36.0), beta_sampled=(24.0, 36.0)),
+                      mpt_mode="dynamic", beta_planted=(18.5, 32.0), beta_sampled=(18.5, 32.0)),
+    # the same batch shape with weaker plants: mean entropy above sigma, so the dynamic gate stays shut
+    "ultra_open": Workload("ultra_open", 5, T=131072, S=1, H=2048, V=151936, dtype="bf16",
+                           lengths="single", segment_len=16384, max_segments=8,
+                           noise="stale:0.02", adv="plus1", planted=0.7, sampled=0.3,
+                           mpt_mode="dynamic", beta_planted=(17.0, 29.0), beta_sampled=(17.0, 29.0)),
 }
 
 

@@ -1,0 +1,134 @@
+"""Parity at the full workload sizes (V = 151936, H = 2048) in the launch configuration that
+bench.py times.  The oracle cannot run 10^14 multiply-adds, so it computes a stratified sample of
+token rows one by one (log-prob, entropy, dHidden row) and a sub-batch for dW; the rest is checked by
+properties that hold at any size (decisions re-derived from the GPU's own log-probs, sequence means,
+dW column sums, independence of dW from the backward panel size)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ulorl_oracle as O
+from paper_2507_19766_b200 import binding as B
+from paper_2507_19766_b200 import synth
+from tests.helpers import TOL_GRAD, TOL_LOGP, both_params, rel_l2
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def stratified_rows(batch, n_random=160, seed=0):
+    wl = batch.workload
+    T = wl.T
+    rng = np.random.default_rng(seed)
+    rows = {0, 1, 127, 128, 129, 255, 256, T - 129, T - 128, T - 1, 16383, 16384, 16385}
+    off = batch.seq_offsets.numpy()
+    for i in range(min(wl.S, 12)):                       # first and last token of some sequences
+        rows.add(int(off[i]))
+        rows.add(int(off[i + 1]) - 1)
+    tg = batch.targets.numpy()
+    tail = np.nonzero(tg >= (wl.V // 256) * 256)[0]       # target inside the last (partial) vocabulary tile
+    rows.update(int(x) for x in tail[:8])
+    ver = batch.segment_version.numpy()
+    for v in np.unique(ver):                             # every policy version
+        idx = np.nonzero(ver == v)[0]
+        rows.update(int(x) for x in rng.choice(idx, size=min(4, idx.size), replace=False))
+    planted = batch.planted_rows
+    for sel in (planted, ~planted):
+        idx = np.nonzero(sel)[0]
+        if idx.size:
+            rows.update(int(x) for x in rng.choice(idx, size=min(n_random // 2, idx.size), replace=False))
+    rows = np.array(sorted(r for r in rows if 0 <= r < T), dtype=np.int64)
+    return rows
+
+
+@pytest.mark.parametrize("name", ["ultra", "qwen", "mixed"])
+def test_full_size_workload_against_sampled_oracle(name):
+    wl = synth.WORKLOADS[name]
+    batch = synth.make_batch(wl, device=DEV)
+    gp, op = both_params(batch)
+    b = batch.to(DEV)
+    ws = B.alloc_workspace(gp, DEV)
+    out = B.token_loss_fwd(gp, b.hidden, b.W, b.targets, b.old_logp, b.segment_version, b.advantages,
+                           b.seq_offsets, workspace=ws)
+    dH, dW = B.token_loss_bwd(gp, b.hidden, b.W, b.targets, out.lse, out.grad_coef, workspace=ws)
+    torch.cuda.synchronize()
+    assert B.check_status(ws) == B.OK
+
+    # ---- sampled rows: log-prob, entropy, lse one by one
+    rows = stratified_rows(batch)
+    rt = torch.from_numpy(rows)
+    W_host = batch.host_f32("W")
+    h_rows = batch.hidden[rt].float().numpy()
+    y_rows = batch.targets[rt].numpy()
+    logp_r, ent_r, lse_r = O.token_stats(h_rows, W_host, y_rows, op.inv_temperature)
+    logp = out.logp.cpu().numpy()
+    ent = out.entropy.cpu().numpy()
+    assert np.abs(logp[rows] - logp_r).max() <= TOL_LOGP
+    assert np.abs(ent[rows] - ent_r).max() <= TOL_LOGP
+    assert np.abs(out.lse.cpu().numpy()[rows] - lse_r).max() <= TOL_LOGP
+    assert np.isfinite(logp).all() and (ent >= 0).all() and (ent <= np.log(wl.V) + 1e-3).all() and (logp <= 1e-6).all()
+
+    # ---- whole batch: sequence means and decisions re-derived by the oracle from the GPU's log-probs
+    off = batch.seq_offsets.numpy()
+    seq_mean, batch_mean = O.sequence_mean_entropy(ent, off)
+    seq_ent = out.seq_entropy.cpu().numpy()[: wl.S]
+    assert np.allclose(seq_ent, seq_mean, rtol=1e-6, atol=1e-9)
+    dec = O.decide(logp, seq_ent, batch.old_logp.numpy(), batch.advantages.numpy(), off,
+                   batch.segment_version.numpy(), op)
+    assert np.array_equal(out.flags.cpu().numpy(), dec["flags"])
+    g = out.grad_coef.cpu().numpy()
+    assert np.allclose(g, dec["grad_coef"], rtol=2e-6, atol=1e-14)
+    st = out.stats_host()
+    for k in ("n_tokens", "n_active", "n_mpt", "n_masked", "n_clip_high", "n_clip_low"):
+        assert st[k] == dec["stats"][k], k
+    assert abs(float(out.loss.cpu()[0]) - dec["loss"]) <= 2e-6 * max(1.0, abs(dec["loss"]))
+    assert abs(st["mean_entropy"] - batch_mean) <= 1e-6
+    if name == "ultra":        # the recipe puts the mean entropy below sigma: the dynamic gate is open
+        assert seq_ent[0] < wl.entropy_target and st["n_masked"] > wl.T // 2 and st["n_active"] > wl.T // 20
+    if name == "mixed":
+        assert st["n_clip_high"] == 0 and st["n_clip_low"] == 0
+
+    # ---- sampled rows of dHidden (rows are independent given g_t)
+    active = rows[g[rows] != 0]
+    assert active.size >= 16
+    sel = np.isin(rows, active)
+    dH_ref, _ = O.backward(h_rows[sel], W_host, y_rows[sel], g[active].astype(np.float64), op.inv_temperature,
+                           want_dW=False)
+    dH_gpu = dH[torch.from_numpy(active).to(DEV)].float().cpu().numpy()
+    assert rel_l2(dH_gpu, dH_ref) <= TOL_GRAD
+    # row by row: no row is off by more than the tolerance times a typical row norm.  (A row whose
+    # target probability is within 1e-5 of one has a gradient ~(1 - p) that float32 cannot resolve
+    # relative to itself; its absolute size is then far below the typical row's.)
+    row_err = np.linalg.norm(dH_gpu - dH_ref, axis=1)
+    row_ref = np.linalg.norm(dH_ref, axis=1)
+    assert (row_err <= 3 * TOL_GRAD * np.maximum(row_ref, np.median(row_ref))).all()
+    inactive = rows[g[rows] == 0]
+    if inactive.size:
+        assert float(dH[torch.from_numpy(inactive).to(DEV)].float().abs().max()) == 0.0
+
+    # ---- dW: properties at full size
+    col = float(dW.double().sum(dim=0).abs().max())
+    coef_sum = float(np.abs(g).sum()) * op.inv_temperature
+    assert col <= 2.0 ** -8 * coef_sum * float(batch.hidden.float().abs().max()) + 1e-12
+    assert torch.isfinite(dW).all()
+    dW_host = dW.cpu()
+    del dW, dH
+    gp2, _ = both_params(batch, bwd_panel_tokens=8192)
+    ws2 = B.alloc_workspace(gp2, DEV)
+    _, dW2 = B.token_loss_bwd(gp2, b.hidden, b.W, b.targets, out.lse, out.grad_coef, workspace=ws2)
+    torch.cuda.synchronize()
+    assert rel_l2(dW2.cpu().numpy(), dW_host.numpy()) <= 1e-4       # same sum, other panel boundaries
+    del dW2, ws2
+
+    # ---- dW: sub-batch of the sampled active rows against the full oracle, same N and same g
+    n_sub = int(active.size)
+    sub = B.Params(T=n_sub, H=wl.H, V=wl.V, num_seqs=1, dtype="bf16", is_mode=wl.is_mode, mpt_mode="off",
+                   norm_tokens=wl.T, current_version=batch.current_version)
+    ta = torch.from_numpy(active).to(DEV)
+    ws3 = B.alloc_workspace(sub, DEV)
+    dH_s, dW_s = B.token_loss_bwd(sub, b.hidden[ta].contiguous(), b.W, b.targets[ta].contiguous(),
+                                  out.lse[ta].contiguous(), out.grad_coef[ta].contiguous(), workspace=ws3)
+    torch.cuda.synchronize()
+    _, dW_ref = O.backward(h_rows[sel], W_host, y_rows[sel], g[active].astype(np.float64), op.inv_temperature)
+    assert rel_l2(dW_s.cpu().numpy(), dW_ref) <= TOL_GRAD
+    assert rel_l2(dH_s.float().cpu().numpy(), dH_ref) <= TOL_GRAD
