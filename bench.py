@@ -24,6 +24,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 from paper_2507_19766_b200 import binding as B  # noqa: E402
+from paper_2507_19766_b200 import dp  # noqa: E402
 from paper_2507_19766_b200 import synth  # noqa: E402
 
 METRIC = "fused loss fwd+bwd tokens/sec at H=2048,V=151936; % of B200 bf16 tensor peak"
@@ -213,7 +214,8 @@ def main():
     gp = B.Params(T=wl.T, H=wl.H, V=wl.V, num_seqs=wl.S, dtype=wl.dtype, is_mode=wl.is_mode, mpt_mode=wl.mpt_mode,
                   clip_eps_low=wl.clip_eps_low, clip_eps_high=wl.clip_eps_high, mpt_tau=wl.mpt_tau,
                   entropy_target=wl.entropy_target, current_version=host_batch.current_version,
-                  bwd_panel_tokens=args.panel)
+                  bwd_panel_tokens=args.panel,
+                  norm_tokens=dp.global_token_count(wl.T, dev) if world > 1 else 0)
     ws = B.alloc_workspace(gp, dev)
     out = B.alloc_fwd_outputs(gp, dev)
     d_hidden = torch.empty_like(b.hidden)
@@ -224,8 +226,8 @@ def main():
                          out=out, workspace=ws)
         B.token_loss_bwd(gp, b.hidden, b.W, b.targets, out.lse, out.grad_coef, d_hidden=d_hidden, d_W=d_W,
                          workspace=ws)
-        if dist is not None:
-            dist.all_reduce(d_W)     # data-parallel exchange: every rank needs the summed head gradient
+        if dist is not None:         # data-parallel exchange: the summed head gradient and loss
+            dp.reduce_step_outputs(d_W, out.loss)
 
     def fence():
         torch.cuda.synchronize()
