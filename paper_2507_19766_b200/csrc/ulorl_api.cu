@@ -4,6 +4,7 @@
 #include <atomic>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -19,6 +20,17 @@ constexpr int kDesignSMs = 148;           // the plan (splits, workspace) is siz
 constexpr int kDefaultPanelTensor = 16384;
 constexpr int kDefaultPanelSimt = 1024;
 constexpr int kRasterGroup = 16;          // row tiles per raster group of the tensor-core kernels
+
+// CTAs per tcgen05.mma: 2 (a CTA pair per 256 x 256 tile, the default) or 1.  The environment
+// variable ULORL_CTA_GROUP=1 selects the single-CTA kernels (read once per process).
+static int cta_group() {
+  static int value = 0;
+  if (value == 0) {
+    const char* e = std::getenv("ULORL_CTA_GROUP");
+    value = (e && e[0] == '1') ? 1 : 2;
+  }
+  return value;
+}
 
 struct Plan {
   bool tensor;            // tensor-core path (bf16) or SIMT path
@@ -56,11 +68,12 @@ static Plan make_plan(const ulorl_params_t* p) {
   Plan pl{};
   pl.tensor = use_tensor_path(p);
   const int T = p->T, V = p->V;
-  const int tile_m = pl.tensor ? kBM : kSimtTile;
+  const int tile_m = pl.tensor ? kBM * cta_group() : kSimtTile;
   const int tile_n = pl.tensor ? kBN : kSimtTile;
+  const int workers = pl.tensor ? kDesignSMs / cta_group() : kDesignSMs;
   const int m_tiles = (T + tile_m - 1) / tile_m;
   const int n_tiles = (V + tile_n - 1) / tile_n;
-  int want = m_tiles > 0 ? (8 * kDesignSMs + m_tiles - 1) / m_tiles : 1;
+  int want = m_tiles > 0 ? (8 * workers + m_tiles - 1) / m_tiles : 1;
   want = want < 1 ? 1 : want;
   want = want > kMaxSplits ? kMaxSplits : want;
   want = want > n_tiles ? n_tiles : want;
@@ -160,12 +173,13 @@ static cudaEvent_t timing_event(int kind) {
   return t.ev[kind][t.used[kind]++];
 }
 
-template <int kMode>
-static int launch_umma(const CUtensorMap& ma, const CUtensorMap& mb, const UmmaArgs& a, cudaStream_t stream) {
+template <int kMode, int kCta>
+static int launch_umma_impl(const CUtensorMap& ma, const CUtensorMap& mb, const UmmaArgs& a, cudaStream_t stream) {
   static bool configured = false;
   static int num_sms = 0;
+  constexpr size_t smem = PipeConfig<kCta>::smem_bytes;
   if (!configured) {
-    if (cudaFuncSetAttribute(umma_kernel<kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUmmaSmemBytes) !=
+    if (cudaFuncSetAttribute(umma_kernel<kMode, kCta>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)
       return ULORL_ERR_CUDA;
     int dev = 0;
@@ -177,17 +191,39 @@ static int launch_umma(const CUtensorMap& ma, const CUtensorMap& mb, const UmmaA
   const int units = (kMode == kModeStats) ? a.m_tiles * a.n_split : a.m_tiles * a.n_tiles;
   if (units <= 0) return ULORL_OK;
   if (kMode != kModeStats && a.group_m <= 0) return ULORL_ERR_INVALID_ARG;
-  const int grid = units < num_sms ? units : num_sms;
+  const int max_workers = num_sms / kCta;
+  const int workers = units < max_workers ? units : max_workers;
   cudaEvent_t e0 = nullptr, e1 = nullptr;
   if (g_timing.enabled) {
     e0 = timing_event(kMode);
     e1 = timing_event(kMode);
     if (e0 && e1) cudaEventRecord(e0, stream);
   }
-  umma_kernel<kMode><<<grid, kUmmaThreads, kUmmaSmemBytes, stream>>>(ma, mb, a);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)(workers * kCta), 1, 1);
+  cfg.blockDim = dim3(kUmmaThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kCta;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t le = cudaLaunchKernelEx(&cfg, umma_kernel<kMode, kCta>, ma, mb, a);
+  if (le != cudaSuccess) {
+    std::fprintf(stderr, "ulorl: cudaLaunchKernelEx failed: %s\n", cudaGetErrorString(le));
+    return ULORL_ERR_CUDA;
+  }
   const int st = check_launch();
   if (e0 && e1) cudaEventRecord(e1, stream);
   return st;
+}
+
+template <int kMode>
+static int launch_umma(const CUtensorMap& ma, const CUtensorMap& mb, const UmmaArgs& a, cudaStream_t stream) {
+  return cta_group() == 2 ? launch_umma_impl<kMode, 2>(ma, mb, a, stream) : launch_umma_impl<kMode, 1>(ma, mb, a, stream);
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -343,11 +379,11 @@ int ulorl_token_loss_fwd(const ulorl_params_t* params, const void* hidden, const
     CUtensorMap map_a, map_b;
     st = make_map_bf16(&map_a, hidden, (uint64_t)T, (uint64_t)H, (uint64_t)H, kBK, kBM);
     if (st != ULORL_OK) return st;
-    st = make_map_bf16(&map_b, W, (uint64_t)V, (uint64_t)H, (uint64_t)H, kBK, kBN);
+    st = make_map_bf16(&map_b, W, (uint64_t)V, (uint64_t)H, (uint64_t)H, kBK, kBN / cta_group());
     if (st != ULORL_OK) return st;
     UmmaArgs a{};
     a.M = T; a.N = V; a.K = H;
-    a.m_tiles = (T + kBM - 1) / kBM;
+    a.m_tiles = (T + kBM * cta_group() - 1) / (kBM * cta_group());
     a.n_tiles = (V + kBN - 1) / kBN;
     a.n_split = pl.n_split;
     a.tiles_per_split = pl.tiles_per_split;
@@ -401,10 +437,11 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
 
   if (pl.tensor) {
     __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(ws + pl.off_dz);
+    const int tile_m = kBM * cta_group();
     CUtensorMap map_hidden_k, map_w_k, map_w_mn, map_hidden_mn;
     st = make_map_bf16(&map_hidden_k, hidden, (uint64_t)T, (uint64_t)H, (uint64_t)H, kBK, kBM);
     if (st != ULORL_OK) return st;
-    st = make_map_bf16(&map_w_k, W, (uint64_t)V, (uint64_t)H, (uint64_t)H, kBK, kBN);
+    st = make_map_bf16(&map_w_k, W, (uint64_t)V, (uint64_t)H, (uint64_t)H, kBK, kBN / cta_group());
     if (st != ULORL_OK) return st;
     st = make_map_bf16(&map_w_mn, W, (uint64_t)V, (uint64_t)H, (uint64_t)H, 64, kBK);
     if (st != ULORL_OK) return st;
@@ -416,7 +453,7 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
       {
         UmmaArgs a{};
         a.M = rows; a.N = V; a.K = H;
-        a.m_tiles = (rows + kBM - 1) / kBM;
+        a.m_tiles = (rows + tile_m - 1) / tile_m;
         a.n_tiles = (int)(pl.dz_ld / kBN) + ((pl.dz_ld % kBN) ? 1 : 0);
         a.group_m = kRasterGroup;
         a.a_mn0 = t0;
@@ -437,7 +474,7 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
       {
         UmmaArgs a{};
         a.M = rows; a.N = H; a.K = V;
-        a.m_tiles = (rows + kBM - 1) / kBM;
+        a.m_tiles = (rows + tile_m - 1) / tile_m;
         a.n_tiles = (H + kBN - 1) / kBN;
         a.group_m = kRasterGroup;
         a.row0 = t0;
@@ -451,7 +488,7 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
       {
         UmmaArgs a{};
         a.M = V; a.N = H; a.K = rows;
-        a.m_tiles = (V + kBM - 1) / kBM;
+        a.m_tiles = (V + tile_m - 1) / tile_m;
         a.n_tiles = (H + kBN - 1) / kBN;
         a.group_m = kRasterGroup;
         a.b_k0 = t0;

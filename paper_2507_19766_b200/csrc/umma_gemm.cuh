@@ -25,14 +25,22 @@ constexpr int kBM = 128;           // accumulator rows (tensor-memory lanes)
 constexpr int kBN = 256;           // accumulator columns
 constexpr int kBK = 64;            // contraction elements per pipeline stage (128 bytes of bf16)
 constexpr int kUmmaK = 16;         // contraction elements per tcgen05.mma
-constexpr int kStages = 4;
 constexpr int kUmmaThreads = 192;
 constexpr int kTmemCols = 512;     // two accumulators of kBN columns
 constexpr uint32_t kABytes = kBM * kBK * 2;
 constexpr uint32_t kBBytes = kBN * kBK * 2;
-constexpr uint32_t kStageBytes = kABytes + kBBytes;
 constexpr uint32_t kChunkBytes = 64 * kBK * 2;   // one MN-major box: 64 k-rows of 64 contiguous elements
-constexpr size_t kUmmaSmemBytes = (size_t)kStages * kStageBytes + 1024;
+
+// Shared-memory ring per CTA.  One CTA alone loads the whole 256-row B tile (48 KB a stage, 4 stages);
+// in a CTA pair each CTA loads its 128 rows of A and half of B (32 KB a stage, 6 stages), and one
+// tcgen05.mma over the pair covers 256 x 256 outputs: a third less L2 traffic per flop and a ring
+// half again as deep in time.
+template <int kCta>
+struct PipeConfig {
+  static constexpr int stages = (kCta == 2) ? 6 : 4;
+  static constexpr uint32_t stage_bytes = kABytes + kBBytes / kCta;
+  static constexpr size_t smem_bytes = (size_t)stages * stage_bytes + 1024;
+};
 constexpr long long kWaitLimitCycles = 4000000000LL;   // about two seconds at the maximum SM clock
 
 enum UmmaMode { kModeStats = 0, kModeDz = 1, kModeDHidden = 2, kModeDW = 3 };
@@ -150,15 +158,21 @@ __device__ __forceinline__ void dz_chunk(const uint32_t (&raw)[32], int nvalid, 
   }
 }
 
-template <int kMode>
+template <int kMode, int kCta>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const UmmaArgs args) {
   using namespace ptx;
+  using Cfg = PipeConfig<kCta>;
+  constexpr bool kPair = (kCta == 2);
   constexpr bool kAmn = ModeTraits<kMode>::a_mn;
   constexpr bool kBmn = ModeTraits<kMode>::b_mn;
+  constexpr int kStagesT = Cfg::stages;
+  constexpr int kBNcta = kBN / kCta;                       // rows of B that this CTA loads
+  constexpr uint32_t kBBytesCta = kBNcta * kBK * 2;
+  constexpr uint32_t kStageBytesCta = kABytes + kBBytesCta;
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bar_full[kStages];
-  __shared__ __align__(8) uint64_t bar_empty[kStages];
+  __shared__ __align__(8) uint64_t bar_full[kStagesT];
+  __shared__ __align__(8) uint64_t bar_empty[kStagesT];
   __shared__ __align__(8) uint64_t bar_tmem_full[2];
   __shared__ __align__(8) uint64_t bar_tmem_empty[2];
   __shared__ uint32_t tmem_base_slot;
@@ -168,16 +182,19 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   const int lane = threadIdx.x & 31;
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   volatile int* abort_p = &abort_flag;
+  const int cta_rank = kPair ? (int)cluster_ctarank() : 0;   // 0 = the CTA that issues the pair's MMAs
+  const int worker = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int n_workers = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < kStagesT; ++s) {
       mbar_init(smem_u32(&bar_full[s]), 1);
       mbar_init(smem_u32(&bar_empty[s]), 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&bar_tmem_full[b]), 1);
-      mbar_init(smem_u32(&bar_tmem_empty[b]), 4);   // one arrival per epilogue warp
+      mbar_init(smem_u32(&bar_tmem_empty[b]), 4 * kCta);   // one arrival per epilogue warp of every CTA
     }
     mbar_fence_init();
     fence_async_proxy();
@@ -187,11 +204,17 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     prefetch_tensormap(&map_b);
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(&tmem_base_slot), kTmemCols);
-    tmem_relinquish();
+    if (kPair) {
+      tmem_alloc_pair(smem_u32(&tmem_base_slot), kTmemCols);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(smem_u32(&tmem_base_slot), kTmemCols);
+      tmem_relinquish();
+    }
   }
   tc_fence_before_sync();
   __syncthreads();
+  if (kPair) cluster_sync_all();                           // the peer's barriers exist before anyone signals them
   tc_fence_after_sync();
   const uint32_t tmem_base = tmem_base_slot;
 
@@ -199,10 +222,10 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   const int n_units = (kMode == kModeStats) ? args.m_tiles * args.n_split : args.m_tiles * args.n_tiles;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ TMA producer (every CTA)
     uint32_t stage = 0, phase = 0;
     uint32_t issued = 0;
-    for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+    for (int unit = worker; unit < n_units; unit += n_workers) {
       int m_tile, n_begin, n_end;
       if (kMode == kModeStats) {
         m_tile = unit / args.n_split;
@@ -212,41 +235,69 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         unit_to_tile(unit, args, m_tile, n_begin);
         n_end = n_begin + 1;
       }
+      const int a_row = args.a_mn0 + (m_tile * kCta + cta_rank) * kBM;
       for (int n_tile = n_begin; n_tile < n_end; ++n_tile) {
+        const int b_row = args.b_mn0 + n_tile * kBN + cta_rank * kBNcta;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait_bounded(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p, kWaitLimitCycles)) goto producer_drain;
           if (lane == 0) {
-            const uint32_t full = smem_u32(&bar_full[stage]);
-            const uint32_t sa = smem_base + stage * kStageBytes;
+            const uint32_t sa = smem_base + stage * kStageBytesCta;
             const uint32_t sb = sa + kABytes;
-            mbar_arrive_expect_tx(full, kStageBytes);
-            if (kAmn) {
+            const int ka = args.a_k0 + kb * kBK, kbb = args.b_k0 + kb * kBK;
+            if (kPair) {
+              // both CTAs' bytes are counted on the issuing CTA's barrier, which alone is armed
+              const uint32_t full = map_to_cta(smem_u32(&bar_full[stage]), 0);
+              if (cta_rank == 0) mbar_arrive_expect_tx(smem_u32(&bar_full[stage]), 2 * kStageBytesCta);
+              if (kAmn) {
 #pragma unroll
-              for (int j = 0; j < kBM / 64; ++j)
-                tma_load_2d(sa + j * kChunkBytes, &map_a, full, args.a_mn0 + m_tile * kBM + j * 64, args.a_k0 + kb * kBK);
-            } else {
-              tma_load_2d(sa, &map_a, full, args.a_k0 + kb * kBK, args.a_mn0 + m_tile * kBM);
-            }
-            if (kBmn) {
+                for (int j = 0; j < kBM / 64; ++j) tma_load_2d_pair(sa + j * kChunkBytes, &map_a, full, a_row + j * 64, ka);
+              } else {
+                tma_load_2d_pair(sa, &map_a, full, ka, a_row);
+              }
+              if (kBmn) {
 #pragma unroll
-              for (int j = 0; j < kBN / 64; ++j)
-                tma_load_2d(sb + j * kChunkBytes, &map_b, full, args.b_mn0 + n_tile * kBN + j * 64, args.b_k0 + kb * kBK);
+                for (int j = 0; j < kBNcta / 64; ++j) tma_load_2d_pair(sb + j * kChunkBytes, &map_b, full, b_row + j * 64, kbb);
+              } else {
+                tma_load_2d_pair(sb, &map_b, full, kbb, b_row);
+              }
             } else {
-              tma_load_2d(sb, &map_b, full, args.b_k0 + kb * kBK, args.b_mn0 + n_tile * kBN);
+              const uint32_t full = smem_u32(&bar_full[stage]);
+              mbar_arrive_expect_tx(full, kStageBytesCta);
+              if (kAmn) {
+#pragma unroll
+                for (int j = 0; j < kBM / 64; ++j) tma_load_2d(sa + j * kChunkBytes, &map_a, full, a_row + j * 64, ka);
+              } else {
+                tma_load_2d(sa, &map_a, full, ka, a_row);
+              }
+              if (kBmn) {
+#pragma unroll
+                for (int j = 0; j < kBNcta / 64; ++j) tma_load_2d(sb + j * kChunkBytes, &map_b, full, b_row + j * 64, kbb);
+              } else {
+                tma_load_2d(sb, &map_b, full, kbb, b_row);
+              }
             }
           }
           __syncwarp();
           ++issued;
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          if (++stage == kStagesT) { stage = 0; phase ^= 1u; }
         }
       }
     }
+    // tail: every slot this CTA filled has been released again, i.e. the MMAs that read this CTA's
+    // shared memory are done and no release signal is still on its way to this CTA
+    {
+      const uint32_t n_tail = issued < (uint32_t)kStagesT ? issued : (uint32_t)kStagesT;
+      for (uint32_t b = 0; b < n_tail; ++b) {
+        if (!mbar_wait_bounded(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p, kWaitLimitCycles)) goto producer_drain;
+        if (++stage == kStagesT) { stage = 0; phase ^= 1u; }
+      }
+    }
   producer_drain:
-    if (*abort_p) {
+    if (*abort_p && cta_rank == 0) {
       // give the copies still in flight a bounded time to land before the block goes away
-      const uint32_t n_back = issued < (uint32_t)kStages ? issued : (uint32_t)kStages;
+      const uint32_t n_back = issued < (uint32_t)kStagesT ? issued : (uint32_t)kStagesT;
       for (uint32_t b = 0; b < n_back; ++b) {
-        if (stage == 0) { stage = kStages; phase ^= 1u; }
+        if (stage == 0) { stage = kStagesT; phase ^= 1u; }
         --stage;
         const long long t0 = clock64();
         while (!mbar_try_wait(smem_u32(&bar_full[stage]), phase) && clock64() - t0 < 200000000LL) {
@@ -254,55 +305,63 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    constexpr uint32_t idesc = make_idesc_bf16(kBM, kBN, kAmn ? 1 : 0, kBmn ? 1 : 0);
-    uint32_t stage = 0, phase = 0;
-    uint32_t acc_iter = 0;
-    for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
-      int n_begin, n_end;
-      if (kMode == kModeStats) {
-        n_begin = (unit % args.n_split) * args.tiles_per_split;
-        n_end = min(args.n_tiles, n_begin + args.tiles_per_split);
-      } else {
-        n_begin = 0;
-        n_end = 1;
-      }
-      for (int n_tile = n_begin; n_tile < n_end; ++n_tile, ++acc_iter) {
-        const uint32_t buf = acc_iter & 1u;
-        const uint32_t buf_phase = (acc_iter >> 1) & 1u;
-        if (!mbar_wait_bounded(smem_u32(&bar_tmem_empty[buf]), buf_phase ^ 1u, abort_p, kWaitLimitCycles)) goto role_done;
-        tc_fence_after_sync();
-        const uint32_t tmem_d = tmem_base + buf * kBN;
-        for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait_bounded(smem_u32(&bar_full[stage]), phase, abort_p, kWaitLimitCycles)) goto role_done;
+    // ------------------------------------------------------------------ MMA issuer (rank 0 of a pair)
+    if (cta_rank == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(kBM * kCta, kBN, kAmn ? 1 : 0, kBmn ? 1 : 0);
+      uint32_t stage = 0, phase = 0;
+      uint32_t acc_iter = 0;
+      for (int unit = worker; unit < n_units; unit += n_workers) {
+        int n_begin, n_end;
+        if (kMode == kModeStats) {
+          n_begin = (unit % args.n_split) * args.tiles_per_split;
+          n_end = min(args.n_tiles, n_begin + args.tiles_per_split);
+        } else {
+          n_begin = 0;
+          n_end = 1;
+        }
+        for (int n_tile = n_begin; n_tile < n_end; ++n_tile, ++acc_iter) {
+          const uint32_t buf = acc_iter & 1u;
+          const uint32_t buf_phase = (acc_iter >> 1) & 1u;
+          if (!mbar_wait_bounded(smem_u32(&bar_tmem_empty[buf]), buf_phase ^ 1u, abort_p, kWaitLimitCycles)) goto role_done;
           tc_fence_after_sync();
-          if (lane == 0) {
-            const uint32_t sa = smem_base + stage * kStageBytes;
-            const uint32_t sb = sa + kABytes;
+          const uint32_t tmem_d = tmem_base + buf * kBN;
+          for (int kb = 0; kb < k_blocks; ++kb) {
+            if (!mbar_wait_bounded(smem_u32(&bar_full[stage]), phase, abort_p, kWaitLimitCycles)) goto role_done;
+            tc_fence_after_sync();
+            if (lane == 0) {
+              const uint32_t sa = smem_base + stage * kStageBytesCta;
+              const uint32_t sb = sa + kABytes;
 #pragma unroll
-            for (int k = 0; k < kBK / kUmmaK; ++k) {
-              // K-major: 16 elements = 32 bytes along the swizzled row; MN-major: 16 k-rows of 128 bytes
-              const uint64_t da = kAmn ? make_smem_desc(sa + k * (kUmmaK * 128), kChunkBytes, 1024)
-                                       : make_smem_desc(sa + k * (kUmmaK * 2), 16, 1024);
-              const uint64_t db = kBmn ? make_smem_desc(sb + k * (kUmmaK * 128), kChunkBytes, 1024)
-                                       : make_smem_desc(sb + k * (kUmmaK * 2), 16, 1024);
-              umma_bf16(tmem_d, da, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+              for (int k = 0; k < kBK / kUmmaK; ++k) {
+                // K-major: 16 elements = 32 bytes along the swizzled row; MN-major: 16 k-rows of 128 bytes
+                const uint64_t da = kAmn ? make_smem_desc(sa + k * (kUmmaK * 128), kChunkBytes, 1024)
+                                         : make_smem_desc(sa + k * (kUmmaK * 2), 16, 1024);
+                const uint64_t db = kBmn ? make_smem_desc(sb + k * (kUmmaK * 128), kChunkBytes, 1024)
+                                         : make_smem_desc(sb + k * (kUmmaK * 2), 16, 1024);
+                if (kPair) umma_bf16_pair(tmem_d, da, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                else umma_bf16(tmem_d, da, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+              }
+              if (kPair) {
+                umma_commit_pair(smem_u32(&bar_empty[stage]), 3);                        // frees the slot in both CTAs
+                if (kb == k_blocks - 1) umma_commit_pair(smem_u32(&bar_tmem_full[buf]), 3);  // accumulator ready
+              } else {
+                umma_commit(smem_u32(&bar_empty[stage]));
+                if (kb == k_blocks - 1) umma_commit(smem_u32(&bar_tmem_full[buf]));
+              }
             }
-            umma_commit(smem_u32(&bar_empty[stage]));                       // frees the smem slot
-            if (kb == k_blocks - 1) umma_commit(smem_u32(&bar_tmem_full[buf]));  // accumulator ready
+            __syncwarp();
+            if (++stage == kStagesT) { stage = 0; phase ^= 1u; }
           }
-          __syncwarp();
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------------ epilogue (warps 2..5, every CTA)
     const int quarter = warp & 3;                       // tensor-memory lanes 32 * quarter ..
     const int row_in_tile = quarter * 32 + lane;
     const float c2 = args.kappa * 1.4426950408889634f;  // exp(kappa a) = 2^(c2 a)
     uint32_t acc_iter = 0;
-    for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+    for (int unit = worker; unit < n_units; unit += n_workers) {
       int m_tile, n_begin, n_end, split = 0;
       if (kMode == kModeStats) {
         m_tile = unit / args.n_split;
@@ -313,7 +372,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         unit_to_tile(unit, args, m_tile, n_begin);
         n_end = n_begin + 1;
       }
-      const int row = m_tile * kBM + row_in_tile;       // row within this launch's M extent
+      const int row = (m_tile * kCta + cta_rank) * kBM + row_in_tile;   // row within this launch's M extent
       const bool row_ok = row < args.M;
       const int grow = args.row0 + row;                 // global token / vocabulary row
 
@@ -406,10 +465,13 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             }
           }
         }
-        // accumulator drained: hand the buffer back to the MMA warp
+        // accumulator drained: hand the buffer back to the MMA warp (of rank 0)
         tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bar_tmem_empty[buf]));
+        if (lane == 0) {
+          if (kPair) mbar_arrive_cluster(map_to_cta(smem_u32(&bar_tmem_empty[buf]), 0));
+          else mbar_arrive(smem_u32(&bar_tmem_empty[buf]));
+        }
       }
 
       if (kMode == kModeStats && row_ok)
@@ -421,9 +483,11 @@ role_done:
   if (*abort_p && lane == 0) atomicOr(args.status, kStatusTimeout);
   tc_fence_before_sync();
   __syncthreads();
+  if (kPair) cluster_sync_all();       // neither CTA leaves while the other may still signal its barriers
   if (warp == 1) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, kTmemCols);
+    if (kPair) tmem_dealloc_pair(tmem_base, kTmemCols);
+    else tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
