@@ -223,30 +223,33 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (every CTA)
-    uint32_t stage = 0, phase = 0;
-    uint32_t issued = 0;
-    for (int unit = worker; unit < n_units; unit += n_workers) {
-      int m_tile, n_begin, n_end;
-      if (kMode == kModeStats) {
-        m_tile = unit / args.n_split;
-        n_begin = (unit % args.n_split) * args.tiles_per_split;
-        n_end = min(args.n_tiles, n_begin + args.tiles_per_split);
-      } else {
-        unit_to_tile(unit, args, m_tile, n_begin);
-        n_end = n_begin + 1;
-      }
-      const int a_row = args.a_mn0 + (m_tile * kCta + cta_rank) * kBM;
-      for (int n_tile = n_begin; n_tile < n_end; ++n_tile) {
-        const int b_row = args.b_mn0 + n_tile * kBN + cta_rank * kBNcta;
-        for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait_bounded(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p, kWaitLimitCycles)) goto producer_drain;
-          if (lane == 0) {
+    // One thread runs the whole loop: nothing in it needs the other lanes, and a warp-wide
+    // rendezvous per k-block would sit on the critical path of the ring.
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      uint32_t issued = 0;
+      const uint32_t full0 = kPair ? map_to_cta(smem_u32(&bar_full[0]), 0) : smem_u32(&bar_full[0]);
+      for (int unit = worker; unit < n_units; unit += n_workers) {
+        int m_tile, n_begin, n_end;
+        if (kMode == kModeStats) {
+          m_tile = unit / args.n_split;
+          n_begin = (unit % args.n_split) * args.tiles_per_split;
+          n_end = min(args.n_tiles, n_begin + args.tiles_per_split);
+        } else {
+          unit_to_tile(unit, args, m_tile, n_begin);
+          n_end = n_begin + 1;
+        }
+        const int a_row = args.a_mn0 + (m_tile * kCta + cta_rank) * kBM;
+        for (int n_tile = n_begin; n_tile < n_end; ++n_tile) {
+          const int b_row = args.b_mn0 + n_tile * kBN + cta_rank * kBNcta;
+          for (int kb = 0; kb < k_blocks; ++kb) {
+            if (!mbar_wait_bounded(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p, kWaitLimitCycles)) goto producer_drain;
             const uint32_t sa = smem_base + stage * kStageBytesCta;
             const uint32_t sb = sa + kABytes;
             const int ka = args.a_k0 + kb * kBK, kbb = args.b_k0 + kb * kBK;
+            const uint32_t full = full0 + stage * (uint32_t)sizeof(uint64_t);
             if (kPair) {
               // both CTAs' bytes are counted on the issuing CTA's barrier, which alone is armed
-              const uint32_t full = map_to_cta(smem_u32(&bar_full[stage]), 0);
               if (cta_rank == 0) mbar_arrive_expect_tx(smem_u32(&bar_full[stage]), 2 * kStageBytesCta);
               if (kAmn) {
 #pragma unroll
@@ -261,7 +264,6 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 tma_load_2d_pair(sb, &map_b, full, kbb, b_row);
               }
             } else {
-              const uint32_t full = smem_u32(&bar_full[stage]);
               mbar_arrive_expect_tx(full, kStageBytesCta);
               if (kAmn) {
 #pragma unroll
@@ -276,85 +278,87 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 tma_load_2d(sb, &map_b, full, kbb, b_row);
               }
             }
-          }
-          __syncwarp();
-          ++issued;
-          if (++stage == kStagesT) { stage = 0; phase ^= 1u; }
-        }
-      }
-    }
-    // tail: every slot this CTA filled has been released again, i.e. the MMAs that read this CTA's
-    // shared memory are done and no release signal is still on its way to this CTA
-    {
-      const uint32_t n_tail = issued < (uint32_t)kStagesT ? issued : (uint32_t)kStagesT;
-      for (uint32_t b = 0; b < n_tail; ++b) {
-        if (!mbar_wait_bounded(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p, kWaitLimitCycles)) goto producer_drain;
-        if (++stage == kStagesT) { stage = 0; phase ^= 1u; }
-      }
-    }
-  producer_drain:
-    if (*abort_p && cta_rank == 0) {
-      // give the copies still in flight a bounded time to land before the block goes away
-      const uint32_t n_back = issued < (uint32_t)kStagesT ? issued : (uint32_t)kStagesT;
-      for (uint32_t b = 0; b < n_back; ++b) {
-        if (stage == 0) { stage = kStagesT; phase ^= 1u; }
-        --stage;
-        const long long t0 = clock64();
-        while (!mbar_try_wait(smem_u32(&bar_full[stage]), phase) && clock64() - t0 < 200000000LL) {
-        }
-      }
-    }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer (rank 0 of a pair)
-    if (cta_rank == 0) {
-      constexpr uint32_t idesc = make_idesc_bf16(kBM * kCta, kBN, kAmn ? 1 : 0, kBmn ? 1 : 0);
-      uint32_t stage = 0, phase = 0;
-      uint32_t acc_iter = 0;
-      for (int unit = worker; unit < n_units; unit += n_workers) {
-        int n_begin, n_end;
-        if (kMode == kModeStats) {
-          n_begin = (unit % args.n_split) * args.tiles_per_split;
-          n_end = min(args.n_tiles, n_begin + args.tiles_per_split);
-        } else {
-          n_begin = 0;
-          n_end = 1;
-        }
-        for (int n_tile = n_begin; n_tile < n_end; ++n_tile, ++acc_iter) {
-          const uint32_t buf = acc_iter & 1u;
-          const uint32_t buf_phase = (acc_iter >> 1) & 1u;
-          if (!mbar_wait_bounded(smem_u32(&bar_tmem_empty[buf]), buf_phase ^ 1u, abort_p, kWaitLimitCycles)) goto role_done;
-          tc_fence_after_sync();
-          const uint32_t tmem_d = tmem_base + buf * kBN;
-          for (int kb = 0; kb < k_blocks; ++kb) {
-            if (!mbar_wait_bounded(smem_u32(&bar_full[stage]), phase, abort_p, kWaitLimitCycles)) goto role_done;
-            tc_fence_after_sync();
-            if (lane == 0) {
-              const uint32_t sa = smem_base + stage * kStageBytesCta;
-              const uint32_t sb = sa + kABytes;
-#pragma unroll
-              for (int k = 0; k < kBK / kUmmaK; ++k) {
-                // K-major: 16 elements = 32 bytes along the swizzled row; MN-major: 16 k-rows of 128 bytes
-                const uint64_t da = kAmn ? make_smem_desc(sa + k * (kUmmaK * 128), kChunkBytes, 1024)
-                                         : make_smem_desc(sa + k * (kUmmaK * 2), 16, 1024);
-                const uint64_t db = kBmn ? make_smem_desc(sb + k * (kUmmaK * 128), kChunkBytes, 1024)
-                                         : make_smem_desc(sb + k * (kUmmaK * 2), 16, 1024);
-                if (kPair) umma_bf16_pair(tmem_d, da, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-                else umma_bf16(tmem_d, da, db, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-              }
-              if (kPair) {
-                umma_commit_pair(smem_u32(&bar_empty[stage]), 3);                        // frees the slot in both CTAs
-                if (kb == k_blocks - 1) umma_commit_pair(smem_u32(&bar_tmem_full[buf]), 3);  // accumulator ready
-              } else {
-                umma_commit(smem_u32(&bar_empty[stage]));
-                if (kb == k_blocks - 1) umma_commit(smem_u32(&bar_tmem_full[buf]));
-              }
-            }
-            __syncwarp();
+            ++issued;
             if (++stage == kStagesT) { stage = 0; phase ^= 1u; }
           }
         }
       }
+      // tail: every slot this CTA filled has been released again, i.e. the MMAs that read this CTA's
+      // shared memory are done and no release signal is still on its way to this CTA
+      {
+        const uint32_t n_tail = issued < (uint32_t)kStagesT ? issued : (uint32_t)kStagesT;
+        for (uint32_t b = 0; b < n_tail; ++b) {
+          if (!mbar_wait_bounded(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p, kWaitLimitCycles)) goto producer_drain;
+          if (++stage == kStagesT) { stage = 0; phase ^= 1u; }
+        }
+      }
+    producer_drain:
+      if (*abort_p && cta_rank == 0) {
+        // give the copies still in flight a bounded time to land before the block goes away
+        const uint32_t n_back = issued < (uint32_t)kStagesT ? issued : (uint32_t)kStagesT;
+        for (uint32_t b = 0; b < n_back; ++b) {
+          if (stage == 0) { stage = kStagesT; phase ^= 1u; }
+          --stage;
+          const long long t0 = clock64();
+          while (!mbar_try_wait(smem_u32(&bar_full[stage]), phase) && clock64() - t0 < 200000000LL) {
+          }
+        }
+      }
     }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (rank 0 of a pair)
+    // One thread, and as little as possible between two tcgen05.mma: descriptors advance by
+    // constants, and the barrier of the next stage is polled right after this stage's MMAs are
+    // queued, so that its latency runs under them.
+    if (cta_rank == 0 && lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(kBM * kCta, kBN, kAmn ? 1 : 0, kBmn ? 1 : 0);
+      // K-major: 16 elements = 32 bytes along the swizzled row; MN-major: 16 k-rows of 128 bytes
+      constexpr uint64_t a_step = (kAmn ? kUmmaK * 128 : kUmmaK * 2) >> 4;
+      constexpr uint64_t b_step = (kBmn ? kUmmaK * 128 : kUmmaK * 2) >> 4;
+      constexpr uint64_t stage_step = kStageBytesCta >> 4;
+      const uint64_t da_base = kAmn ? make_smem_desc(smem_base, kChunkBytes, 1024) : make_smem_desc(smem_base, 16, 1024);
+      const uint64_t db_base = kBmn ? make_smem_desc(smem_base + kABytes, kChunkBytes, 1024)
+                                    : make_smem_desc(smem_base + kABytes, 16, 1024);
+      uint32_t stage = 0, phase = 0;
+      uint32_t acc_iter = 0;
+      bool ready = false;
+      for (int unit = worker; unit < n_units; unit += n_workers) {
+        int n_tiles_here = 1;
+        if (kMode == kModeStats) {
+          const int n_begin = (unit % args.n_split) * args.tiles_per_split;
+          n_tiles_here = min(args.n_tiles, n_begin + args.tiles_per_split) - n_begin;
+        }
+        for (int t = 0; t < n_tiles_here; ++t, ++acc_iter) {
+          const uint32_t buf = acc_iter & 1u;
+          const uint32_t buf_phase = (acc_iter >> 1) & 1u;
+          if (!mbar_wait_bounded(smem_u32(&bar_tmem_empty[buf]), buf_phase ^ 1u, abort_p, kWaitLimitCycles)) goto mma_done;
+          const uint32_t tmem_d = tmem_base + buf * kBN;
+          for (int kb = 0; kb < k_blocks; ++kb) {
+            if (!ready && !mbar_wait_bounded(smem_u32(&bar_full[stage]), phase, abort_p, kWaitLimitCycles)) goto mma_done;
+            tc_fence_after_sync();
+            const uint64_t da = da_base + stage * stage_step;
+            const uint64_t db = db_base + stage * stage_step;
+#pragma unroll
+            for (int k = 0; k < kBK / kUmmaK; ++k) {
+              if (kPair) umma_bf16_pair(tmem_d, da + k * a_step, db + k * b_step, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+              else umma_bf16(tmem_d, da + k * a_step, db + k * b_step, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            }
+            if (kPair) {
+              umma_commit_pair(smem_u32(&bar_empty[stage]), 3);                        // frees the slot in both CTAs
+              if (kb == k_blocks - 1) umma_commit_pair(smem_u32(&bar_tmem_full[buf]), 3);  // accumulator ready
+            } else {
+              umma_commit(smem_u32(&bar_empty[stage]));
+              if (kb == k_blocks - 1) umma_commit(smem_u32(&bar_tmem_full[buf]));
+            }
+            if (++stage == kStagesT) { stage = 0; phase ^= 1u; }
+            ready = mbar_try_wait(smem_u32(&bar_full[stage]), phase);
+          }
+        }
+      }
+    mma_done:;
+    }
+    __syncwarp();
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..5, every CTA)
     const int quarter = warp & 3;                       // tensor-memory lanes 32 * quarter ..
