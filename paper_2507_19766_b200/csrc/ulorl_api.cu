@@ -17,9 +17,11 @@ namespace ulorl {
 
 static std::atomic<long long> g_launches{0};
 constexpr int kDesignSMs = 148;           // the plan (splits, workspace) is sized for a B200
-constexpr int kDefaultPanelTensor = 16384;
+constexpr int kDefaultPanelTensor = 16384;       // single-CTA kernels
+constexpr int kDefaultPanelPair = 18944;         // CTA pairs: 74 pairs x 256 tokens, whole waves of d_hidden units
 constexpr int kDefaultPanelSimt = 1024;
-constexpr int kRasterGroup = 16;          // row tiles per raster group of the tensor-core kernels
+constexpr int kRasterGroup = 16;          // dz: row tiles per raster group (m fastest inside a group)
+constexpr int kGradRasterGroup = 1;       // d_hidden, d_W: column blocks of one row tile run side by side, so its A stream is read once
 
 // CTAs per tcgen05.mma: 2 (a CTA pair per 256 x 256 tile, the default) or 1.  The environment
 // variable ULORL_CTA_GROUP=1 selects the single-CTA kernels (read once per process).
@@ -79,7 +81,8 @@ static Plan make_plan(const ulorl_params_t* p) {
   want = want > n_tiles ? n_tiles : want;
   pl.tiles_per_split = (n_tiles + want - 1) / want;
   pl.n_split = (n_tiles + pl.tiles_per_split - 1) / pl.tiles_per_split;
-  int panel = p->bwd_panel_tokens > 0 ? p->bwd_panel_tokens : (pl.tensor ? kDefaultPanelTensor : kDefaultPanelSimt);
+  int panel = p->bwd_panel_tokens > 0 ? p->bwd_panel_tokens
+                                      : (pl.tensor ? (cta_group() == 2 ? kDefaultPanelPair : kDefaultPanelTensor) : kDefaultPanelSimt);
   panel = (panel + kBM - 1) / kBM * kBM;
   const int t_round = (T + kBM - 1) / kBM * kBM;
   if (panel > t_round) panel = t_round;
@@ -173,13 +176,13 @@ static cudaEvent_t timing_event(int kind) {
   return t.ev[kind][t.used[kind]++];
 }
 
-template <int kMode, int kCta>
+template <int kMode, int kCta, int kAcc>
 static int launch_umma_impl(const CUtensorMap& ma, const CUtensorMap& mb, const UmmaArgs& a, cudaStream_t stream) {
   static bool configured = false;
   static int num_sms = 0;
-  constexpr size_t smem = PipeConfig<kCta>::smem_bytes;
+  constexpr size_t smem = PipeConfig<kCta, kAcc>::smem_bytes;
   if (!configured) {
-    if (cudaFuncSetAttribute(umma_kernel<kMode, kCta>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+    if (cudaFuncSetAttribute(umma_kernel<kMode, kCta, kAcc>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)
       return ULORL_ERR_CUDA;
     int dev = 0;
@@ -211,7 +214,7 @@ static int launch_umma_impl(const CUtensorMap& ma, const CUtensorMap& mb, const 
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  const cudaError_t le = cudaLaunchKernelEx(&cfg, umma_kernel<kMode, kCta>, ma, mb, a);
+  const cudaError_t le = cudaLaunchKernelEx(&cfg, umma_kernel<kMode, kCta, kAcc>, ma, mb, a);
   if (le != cudaSuccess) {
     std::fprintf(stderr, "ulorl: cudaLaunchKernelEx failed: %s\n", cudaGetErrorString(le));
     return ULORL_ERR_CUDA;
@@ -221,9 +224,15 @@ static int launch_umma_impl(const CUtensorMap& ma, const CUtensorMap& mb, const 
   return st;
 }
 
+// Accumulators per unit: the gradient contractions on CTA pairs use two (256 x 512 outputs a unit).
+template <int kMode>
+static constexpr int acc_per_unit_pair() { return (kMode == kModeDHidden || kMode == kModeDW) ? 2 : 1; }
+static int grad_unit_cols() { return cta_group() == 2 ? 2 * kBN : kBN; }
+
 template <int kMode>
 static int launch_umma(const CUtensorMap& ma, const CUtensorMap& mb, const UmmaArgs& a, cudaStream_t stream) {
-  return cta_group() == 2 ? launch_umma_impl<kMode, 2>(ma, mb, a, stream) : launch_umma_impl<kMode, 1>(ma, mb, a, stream);
+  return cta_group() == 2 ? launch_umma_impl<kMode, 2, acc_per_unit_pair<kMode>()>(ma, mb, a, stream)
+                          : launch_umma_impl<kMode, 1, 1>(ma, mb, a, stream);
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -475,8 +484,8 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
         UmmaArgs a{};
         a.M = rows; a.N = H; a.K = V;
         a.m_tiles = (rows + tile_m - 1) / tile_m;
-        a.n_tiles = (H + kBN - 1) / kBN;
-        a.group_m = kRasterGroup;
+        a.n_tiles = (H + grad_unit_cols() - 1) / grad_unit_cols();
+        a.group_m = kGradRasterGroup;
         a.row0 = t0;
         a.d_hidden = static_cast<__nv_bfloat16*>(d_hidden);
         a.out_ld = (size_t)H;
@@ -489,8 +498,8 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
         UmmaArgs a{};
         a.M = V; a.N = H; a.K = rows;
         a.m_tiles = (V + tile_m - 1) / tile_m;
-        a.n_tiles = (H + kBN - 1) / kBN;
-        a.group_m = kRasterGroup;
+        a.n_tiles = (H + grad_unit_cols() - 1) / grad_unit_cols();
+        a.group_m = kGradRasterGroup;
         a.b_k0 = t0;
         a.d_W = d_W;
         a.out_ld = (size_t)H;

@@ -33,12 +33,15 @@ constexpr uint32_t kChunkBytes = 64 * kBK * 2;   // one MN-major box: 64 k-rows 
 
 // Shared-memory ring per CTA.  One CTA alone loads the whole 256-row B tile (48 KB a stage, 4 stages);
 // in a CTA pair each CTA loads its 128 rows of A and half of B (32 KB a stage, 6 stages), and one
-// tcgen05.mma over the pair covers 256 x 256 outputs: a third less L2 traffic per flop and a ring
-// half again as deep in time.
-template <int kCta>
+// tcgen05.mma over the pair covers 256 x 256 outputs: a third less L2 traffic per flop.  With two
+// accumulators per unit (kAcc = 2) a pair covers 256 x 512 outputs per k-block: A is loaded once
+// for both column blocks (48 KB a stage, 4 stages), eight MMAs are queued per barrier round trip,
+// and tensor memory is used as one 512-column buffer, so the epilogue does not overlap the next
+// unit -- right for the gradient contractions, whose reduction runs over 10^4..10^5 elements.
+template <int kCta, int kAcc>
 struct PipeConfig {
-  static constexpr int stages = (kCta == 2) ? 6 : 4;
-  static constexpr uint32_t stage_bytes = kABytes + kBBytes / kCta;
+  static constexpr uint32_t stage_bytes = kABytes + kAcc * kBBytes / kCta;
+  static constexpr int stages = (int)(196608u / stage_bytes);
   static constexpr size_t smem_bytes = (size_t)stages * stage_bytes + 1024;
 };
 constexpr long long kWaitLimitCycles = 4000000000LL;   // about two seconds at the maximum SM clock
@@ -47,7 +50,7 @@ enum UmmaMode { kModeStats = 0, kModeDz = 1, kModeDHidden = 2, kModeDW = 3 };
 
 struct UmmaArgs {
   int M, N, K;              // extents of the contraction handled by this launch (valid elements)
-  int m_tiles, n_tiles;     // ceil(M / kBM), ceil(N / kBN)
+  int m_tiles, n_tiles;     // ceil(M / rows per unit), ceil(N / columns per unit)
   int n_split;              // kModeStats: vocabulary splits; a unit is (token tile, split)
   int tiles_per_split;
   int group_m;              // other modes: token tiles per raster group (tiles of a group run m-fastest)
@@ -158,18 +161,21 @@ __device__ __forceinline__ void dz_chunk(const uint32_t (&raw)[32], int nvalid, 
   }
 }
 
-template <int kMode, int kCta>
+template <int kMode, int kCta, int kAcc>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const UmmaArgs args) {
   using namespace ptx;
-  using Cfg = PipeConfig<kCta>;
+  using Cfg = PipeConfig<kCta, kAcc>;
+  static_assert(kAcc == 1 || (kCta == 2 && (kMode == kModeDHidden || kMode == kModeDW)), "two accumulators: gradient modes, CTA pairs");
+  constexpr int kBufs = 2 / kAcc;                          // tensor-memory buffers of kAcc accumulators
+  constexpr int kUnitN = kBN * kAcc;                       // output columns per unit
   constexpr bool kPair = (kCta == 2);
   constexpr bool kAmn = ModeTraits<kMode>::a_mn;
   constexpr bool kBmn = ModeTraits<kMode>::b_mn;
   constexpr int kStagesT = Cfg::stages;
   constexpr int kBNcta = kBN / kCta;                       // rows of B that this CTA loads
   constexpr uint32_t kBBytesCta = kBNcta * kBK * 2;
-  constexpr uint32_t kStageBytesCta = kABytes + kBBytesCta;
+  constexpr uint32_t kStageBytesCta = kABytes + kAcc * kBBytesCta;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[kStagesT];
   __shared__ __align__(8) uint64_t bar_empty[kStagesT];
@@ -192,7 +198,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       mbar_init(smem_u32(&bar_full[s]), 1);
       mbar_init(smem_u32(&bar_empty[s]), 1);
     }
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < 2; ++b) {   // with kAcc = 2 only entry 0 is used
       mbar_init(smem_u32(&bar_tmem_full[b]), 1);
       mbar_init(smem_u32(&bar_tmem_empty[b]), 4 * kCta);   // one arrival per epilogue warp of every CTA
     }
@@ -241,7 +247,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
         const int a_row = args.a_mn0 + (m_tile * kCta + cta_rank) * kBM;
         for (int n_tile = n_begin; n_tile < n_end; ++n_tile) {
-          const int b_row = args.b_mn0 + n_tile * kBN + cta_rank * kBNcta;
+          const int b_row = args.b_mn0 + n_tile * kUnitN + cta_rank * kBNcta;   // + kBN per further accumulator
           for (int kb = 0; kb < k_blocks; ++kb) {
             if (!mbar_wait_bounded(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p, kWaitLimitCycles)) goto producer_drain;
             const uint32_t sa = smem_base + stage * kStageBytesCta;
@@ -257,11 +263,15 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
               } else {
                 tma_load_2d_pair(sa, &map_a, full, ka, a_row);
               }
-              if (kBmn) {
 #pragma unroll
-                for (int j = 0; j < kBNcta / 64; ++j) tma_load_2d_pair(sb + j * kChunkBytes, &map_b, full, b_row + j * 64, kbb);
-              } else {
-                tma_load_2d_pair(sb, &map_b, full, kbb, b_row);
+              for (int q = 0; q < kAcc; ++q) {
+                if (kBmn) {
+#pragma unroll
+                  for (int j = 0; j < kBNcta / 64; ++j)
+                    tma_load_2d_pair(sb + q * kBBytesCta + j * kChunkBytes, &map_b, full, b_row + q * kBN + j * 64, kbb);
+                } else {
+                  tma_load_2d_pair(sb + q * kBBytesCta, &map_b, full, kbb, b_row + q * kBN);
+                }
               }
             } else {
               mbar_arrive_expect_tx(full, kStageBytesCta);
@@ -330,19 +340,23 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           n_tiles_here = min(args.n_tiles, n_begin + args.tiles_per_split) - n_begin;
         }
         for (int t = 0; t < n_tiles_here; ++t, ++acc_iter) {
-          const uint32_t buf = acc_iter & 1u;
-          const uint32_t buf_phase = (acc_iter >> 1) & 1u;
+          const uint32_t buf = acc_iter % kBufs;
+          const uint32_t buf_phase = (acc_iter / kBufs) & 1u;
           if (!mbar_wait_bounded(smem_u32(&bar_tmem_empty[buf]), buf_phase ^ 1u, abort_p, kWaitLimitCycles)) goto mma_done;
-          const uint32_t tmem_d = tmem_base + buf * kBN;
+          const uint32_t tmem_d = tmem_base + buf * kUnitN;
           for (int kb = 0; kb < k_blocks; ++kb) {
             if (!ready && !mbar_wait_bounded(smem_u32(&bar_full[stage]), phase, abort_p, kWaitLimitCycles)) goto mma_done;
             tc_fence_after_sync();
             const uint64_t da = da_base + stage * stage_step;
             const uint64_t db = db_base + stage * stage_step;
 #pragma unroll
-            for (int k = 0; k < kBK / kUmmaK; ++k) {
-              if (kPair) umma_bf16_pair(tmem_d, da + k * a_step, db + k * b_step, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-              else umma_bf16(tmem_d, da + k * a_step, db + k * b_step, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            for (int q = 0; q < kAcc; ++q) {
+#pragma unroll
+              for (int k = 0; k < kBK / kUmmaK; ++k) {
+                const uint64_t dbq = db + q * (uint64_t)(kBBytesCta >> 4) + k * b_step;
+                if (kPair) umma_bf16_pair(tmem_d + q * kBN, da + k * a_step, dbq, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                else umma_bf16(tmem_d + q * kBN, da + k * a_step, dbq, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+              }
             }
             if (kPair) {
               umma_commit_pair(smem_u32(&bar_empty[stage]), 3);                        // frees the slot in both CTAs
@@ -402,14 +416,14 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       }
 
       for (int n_tile = n_begin; n_tile < n_end; ++n_tile, ++acc_iter) {
-        const uint32_t buf = acc_iter & 1u;
-        const uint32_t buf_phase = (acc_iter >> 1) & 1u;
+        const uint32_t buf = acc_iter % kBufs;
+        const uint32_t buf_phase = (acc_iter / kBufs) & 1u;
         if (!mbar_wait_bounded(smem_u32(&bar_tmem_full[buf]), buf_phase, abort_p, kWaitLimitCycles)) goto role_done;
         tc_fence_after_sync();
-        const uint32_t taddr = tmem_base + buf * kBN + ((uint32_t)(quarter * 32) << 16);
-        const int col_base = n_tile * kBN;
+        const uint32_t taddr = tmem_base + buf * kUnitN + ((uint32_t)(quarter * 32) << 16);
+        const int col_base = n_tile * kUnitN;
 #pragma unroll 1
-        for (int c = 0; c < kBN / 32; ++c) {
+        for (int c = 0; c < kUnitN / 32; ++c) {
           const int col0 = col_base + c * 32;
           if (kMode != kModeDz && col0 >= args.N) break;       // whole chunk beyond the valid columns
           if (kMode == kModeDz && col0 >= args.dz_cols) break;
