@@ -139,15 +139,15 @@ static EncodeTiledFn get_encode_fn() {
 
 // bf16 matrix [rows][cols] with `ld` elements between rows; box = box_cols x box_rows, 128-byte swizzle,
 // out-of-range elements read as zero.
-static int make_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
-                         uint32_t box_cols, uint32_t box_rows) {
+static int make_map(CUtensorMap* map, CUtensorMapDataType dtype, size_t elem_bytes, const void* base, uint64_t rows,
+                    uint64_t cols, uint64_t ld, uint32_t box_cols, uint32_t box_rows) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return ULORL_ERR_CUDA;
   const cuuint64_t dims[2] = {cols, rows};
-  const cuuint64_t strides[1] = {ld * 2};
+  const cuuint64_t strides[1] = {ld * elem_bytes};
   const cuuint32_t box[2] = {box_cols, box_rows};
   const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  const CUresult r = fn(map, dtype, 2, const_cast<void*>(base), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
@@ -155,6 +155,11 @@ static int make_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uint
     return ULORL_ERR_CUDA;
   }
   return ULORL_OK;
+}
+
+static int make_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
+                         uint32_t box_cols, uint32_t box_rows) {
+  return make_map(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, rows, cols, ld, box_cols, box_rows);
 }
 
 // Optional per-kernel timing of the tensor-core launches: when enabled, an event pair brackets
@@ -177,7 +182,8 @@ static cudaEvent_t timing_event(int kind) {
 }
 
 template <int kMode, int kCta, int kAcc>
-static int launch_umma_impl(const CUtensorMap& ma, const CUtensorMap& mb, const UmmaArgs& a, cudaStream_t stream) {
+static int launch_umma_impl(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const UmmaArgs& a,
+                            cudaStream_t stream) {
   static bool configured = false;
   static int num_sms = 0;
   constexpr size_t smem = PipeConfig<kCta, kAcc>::smem_bytes;
@@ -214,7 +220,7 @@ static int launch_umma_impl(const CUtensorMap& ma, const CUtensorMap& mb, const 
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  const cudaError_t le = cudaLaunchKernelEx(&cfg, umma_kernel<kMode, kCta, kAcc>, ma, mb, a);
+  const cudaError_t le = cudaLaunchKernelEx(&cfg, umma_kernel<kMode, kCta, kAcc>, ma, mb, mc, a);
   if (le != cudaSuccess) {
     std::fprintf(stderr, "ulorl: cudaLaunchKernelEx failed: %s\n", cudaGetErrorString(le));
     return ULORL_ERR_CUDA;
@@ -229,10 +235,12 @@ template <int kMode>
 static constexpr int acc_per_unit_pair() { return (kMode == kModeDHidden || kMode == kModeDW) ? 2 : 1; }
 static int grad_unit_cols() { return cta_group() == 2 ? 2 * kBN : kBN; }
 
+// mc is the output tensor map of the d_W kernel; the other kernels get any valid map and ignore it.
 template <int kMode>
-static int launch_umma(const CUtensorMap& ma, const CUtensorMap& mb, const UmmaArgs& a, cudaStream_t stream) {
-  return cta_group() == 2 ? launch_umma_impl<kMode, 2, acc_per_unit_pair<kMode>()>(ma, mb, a, stream)
-                          : launch_umma_impl<kMode, 1, 1>(ma, mb, a, stream);
+static int launch_umma(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const UmmaArgs& a,
+                       cudaStream_t stream) {
+  return cta_group() == 2 ? launch_umma_impl<kMode, 2, acc_per_unit_pair<kMode>()>(ma, mb, mc, a, stream)
+                          : launch_umma_impl<kMode, 1, 1>(ma, mb, mc, a, stream);
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -402,7 +410,7 @@ int ulorl_token_loss_fwd(const ulorl_params_t* params, const void* hidden, const
     a.acc_y = acc_y;
     a.T_total = T;
     a.status = status;
-    st = launch_umma<kModeStats>(map_a, map_b, a, stream);
+    st = launch_umma<kModeStats>(map_a, map_b, map_a, a, stream);
     if (st != ULORL_OK) return st;
   } else {
     const dim3 grid((T + kSimtTile - 1) / kSimtTile, pl.n_split);
@@ -456,6 +464,9 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
     if (st != ULORL_OK) return st;
     st = make_map_bf16(&map_hidden_mn, hidden, (uint64_t)T, (uint64_t)H, (uint64_t)H, 64, kBK);
     if (st != ULORL_OK) return st;
+    CUtensorMap map_dw_out;   // d_W as the target of 128-row x 32-column float tiles
+    st = make_map(&map_dw_out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, d_W, (uint64_t)V, (uint64_t)H, (uint64_t)H, 32, kBM);
+    if (st != ULORL_OK) return st;
     for (int t0 = 0, panel = 0; t0 < T; t0 += pl.panel_tokens, ++panel) {
       const int rows = (T - t0) < pl.panel_tokens ? (T - t0) : pl.panel_tokens;
       // dz panel: recompute logits, softmax minus one-hot scaled by the token's coefficient
@@ -471,7 +482,7 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
         a.targets = targets; a.lse = lse; a.grad_coef = grad_coef; a.grad_loss = grad_loss;
         a.dz = dz; a.dz_ld = pl.dz_ld; a.dz_cols = (int)pl.dz_ld;
         a.status = status;
-        st = launch_umma<kModeDz>(map_hidden_k, map_w_k, a, stream);
+        st = launch_umma<kModeDz>(map_hidden_k, map_w_k, map_w_k, a, stream);
         if (st != ULORL_OK) return st;
       }
       CUtensorMap map_dz_k, map_dz_mn;
@@ -490,7 +501,7 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
         a.d_hidden = static_cast<__nv_bfloat16*>(d_hidden);
         a.out_ld = (size_t)H;
         a.status = status;
-        st = launch_umma<kModeDHidden>(map_dz_k, map_w_mn, a, stream);
+        st = launch_umma<kModeDHidden>(map_dz_k, map_w_mn, map_w_mn, a, stream);
         if (st != ULORL_OK) return st;
       }
       // d_W[v, h] (+)= sum_m dz[m, v] hidden[t0 + m, h]
@@ -505,7 +516,7 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
         a.out_ld = (size_t)H;
         a.accumulate = (panel > 0 || params->dw_accumulate) ? 1 : 0;
         a.status = status;
-        st = launch_umma<kModeDW>(map_dz_mn, map_hidden_mn, a, stream);
+        st = launch_umma<kModeDW>(map_dz_mn, map_hidden_mn, map_dw_out, a, stream);
         if (st != ULORL_OK) return st;
       }
     }

@@ -38,11 +38,15 @@ constexpr uint32_t kChunkBytes = 64 * kBK * 2;   // one MN-major box: 64 k-rows 
 // for both column blocks (48 KB a stage, 4 stages), eight MMAs are queued per barrier round trip,
 // and tensor memory is used as one 512-column buffer, so the epilogue does not overlap the next
 // unit -- right for the gradient contractions, whose reduction runs over 10^4..10^5 elements.
+// Two staging tiles (128 rows x 128 bytes each, 128-byte swizzle) through which the d_W epilogue
+// hands 32-column chunks of the accumulator to TMA store / reduce-add.
+constexpr uint32_t kOutStageBytes = kBM * 128;
+
 template <int kCta, int kAcc>
 struct PipeConfig {
   static constexpr uint32_t stage_bytes = kABytes + kAcc * kBBytes / kCta;
   static constexpr int stages = (int)(196608u / stage_bytes);
-  static constexpr size_t smem_bytes = (size_t)stages * stage_bytes + 1024;
+  static constexpr size_t smem_bytes = (size_t)stages * stage_bytes + 1024 + 2 * kOutStageBytes;
 };
 constexpr long long kWaitLimitCycles = 4000000000LL;   // about two seconds at the maximum SM clock
 
@@ -163,7 +167,8 @@ __device__ __forceinline__ void dz_chunk(const uint32_t (&raw)[32], int nvalid, 
 
 template <int kMode, int kCta, int kAcc>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
-umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const UmmaArgs args) {
+umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+            const __grid_constant__ CUtensorMap map_c, const UmmaArgs args) {
   using namespace ptx;
   using Cfg = PipeConfig<kCta, kAcc>;
   static_assert(kAcc == 1 || (kCta == 2 && (kMode == kModeDHidden || kMode == kModeDW)), "two accumulators: gradient modes, CTA pairs");
@@ -418,19 +423,19 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       for (int n_tile = n_begin; n_tile < n_end; ++n_tile, ++acc_iter) {
         const uint32_t buf = acc_iter % kBufs;
         const uint32_t buf_phase = (acc_iter / kBufs) & 1u;
+        const int col_base = n_tile * kUnitN;
         if (!mbar_wait_bounded(smem_u32(&bar_tmem_full[buf]), buf_phase, abort_p, kWaitLimitCycles)) goto role_done;
         tc_fence_after_sync();
         const uint32_t taddr = tmem_base + buf * kUnitN + ((uint32_t)(quarter * 32) << 16);
-        const int col_base = n_tile * kUnitN;
 #pragma unroll 1
         for (int c = 0; c < kUnitN / 32; ++c) {
           const int col0 = col_base + c * 32;
           if (kMode != kModeDz && col0 >= args.N) break;       // whole chunk beyond the valid columns
           if (kMode == kModeDz && col0 >= args.dz_cols) break;
+          const int nvalid = min(32, args.N - col0);           // may be <= 0 only in kModeDz padding
           uint32_t raw[32];
           tmem_ld_32x32(taddr + c * 32, raw);
           tmem_ld_wait();
-          const int nvalid = min(32, args.N - col0);           // may be <= 0 only in kModeDz padding
 
           if (kMode == kModeStats) {
             if (nvalid >= 32) stats_chunk<true>(raw, 32, c2, run_m, run_s, run_u);
@@ -465,21 +470,28 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
               for (int q = 0; q < 4; ++q)
                 if (q * 8 < nvalid) dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
             }
-          } else {  // kModeDW
-            if (row_ok) {
-              float4* dst = reinterpret_cast<float4*>(args.d_W + (size_t)grow * args.out_ld + col0);
+          } else {  // kModeDW: swizzled staging tile, then one TMA store (first panel) or reduce-add
+            const uint32_t out_buf = smem_base + kStagesT * kStageBytesCta + (uint32_t)(c & 1) * kOutStageBytes;
+            const bool issuer = (threadIdx.x == 64);             // first thread of the epilogue warps
+            if (issuer) bulk_wait_read_le1();                    // the copy that last read this tile is done with it
+            epilogue_bar_sync();
+            const uint32_t row_addr = out_buf + (uint32_t)row_in_tile * 128u;
 #pragma unroll
-              for (int q = 0; q < 8; ++q) {
-                if (q * 4 < nvalid) {
-                  float4 v = make_float4(__uint_as_float(raw[4 * q]), __uint_as_float(raw[4 * q + 1]),
-                                         __uint_as_float(raw[4 * q + 2]), __uint_as_float(raw[4 * q + 3]));
-                  if (args.accumulate) {
-                    const float4 o = dst[q];
-                    v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-                  }
-                  dst[q] = v;
-                }
+            for (int q = 0; q < 8; ++q) {
+              const uint32_t dst = row_addr + ((uint32_t)(q ^ (row_in_tile & 7)) << 4);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(raw[4 * q]), "r"(raw[4 * q + 1]),
+                           "r"(raw[4 * q + 2]), "r"(raw[4 * q + 3])
+                           : "memory");
+            }
+            fence_async_proxy();
+            epilogue_bar_sync();
+            if (issuer) {
+              const int tile_row = (m_tile * kCta + cta_rank) * kBM;      // rows past M never reach memory
+              if (tile_row < args.M) {
+                if (args.accumulate) tma_reduce_add_2d(&map_c, out_buf, col0, args.row0 + tile_row);
+                else tma_store_2d(&map_c, out_buf, col0, args.row0 + tile_row);
               }
+              bulk_commit_group();
             }
           }
         }
@@ -498,6 +510,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   }
 
 role_done:
+  if (kMode == kModeDW && threadIdx.x == 64) bulk_wait_all();   // the tile copies have left shared memory and landed
   if (*abort_p && lane == 0) atomicOr(args.status, kStatusTimeout);
   tc_fence_before_sync();
   __syncthreads();
