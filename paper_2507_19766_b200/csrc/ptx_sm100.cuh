@@ -55,12 +55,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Wait for the phase of `parity` to complete, giving up after `limit_cycles` SM clocks or
 // as soon as another thread of the block has raised `*abort_flag`.  On giving up the flag is
 // raised so that every role of the block leaves its loop.
+template <bool kBackoff = false>
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                                   long long limit_cycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
+    if (kBackoff) __nanosleep(200);      // waits that are long by design: leave the issue slots alone
     if ((it & 63u) == 0u) {
       if (*abort_flag) return false;
       if (clock64() - t0 > limit_cycles) {

@@ -186,7 +186,7 @@ static int launch_umma_impl(const CUtensorMap& ma, const CUtensorMap& mb, const 
                             cudaStream_t stream) {
   static bool configured = false;
   static int num_sms = 0;
-  constexpr size_t smem = PipeConfig<kCta, kAcc>::smem_bytes;
+  constexpr size_t smem = PipeConfig<kCta, kAcc, KAtoms<kMode, kCta>::value>::smem_bytes;
   if (!configured) {
     if (cudaFuncSetAttribute(umma_kernel<kMode, kCta, kAcc>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)

@@ -42,9 +42,15 @@ constexpr uint32_t kChunkBytes = 64 * kBK * 2;   // one MN-major box: 64 k-rows 
 // hands 32-column chunks of the accumulator to TMA store / reduce-add.
 constexpr uint32_t kOutStageBytes = kBM * 128;
 
-template <int kCta, int kAcc>
+// A stage holds kKA "atoms" of 64 contraction elements (one 128-byte swizzle span each); the two
+// logits kernels use two atoms a stage, so that eight MMAs are queued per barrier round trip there too.
+template <int kMode, int kCta>
+struct KAtoms { static constexpr int value = (kCta == 2 && (kMode == 0 || kMode == 1)) ? 2 : 1; };
+
+template <int kCta, int kAcc, int kKA>
 struct PipeConfig {
-  static constexpr uint32_t stage_bytes = kABytes + kAcc * kBBytes / kCta;
+  static constexpr uint32_t atom_bytes = kABytes + kAcc * kBBytes / kCta;
+  static constexpr uint32_t stage_bytes = kKA * atom_bytes;
   static constexpr int stages = (int)(196608u / stage_bytes);
   static constexpr size_t smem_bytes = (size_t)stages * stage_bytes + 1024 + 2 * kOutStageBytes;
 };
@@ -170,7 +176,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const __grid_constant__ CUtensorMap map_c, const UmmaArgs args) {
   using namespace ptx;
-  using Cfg = PipeConfig<kCta, kAcc>;
+  constexpr int kKA = KAtoms<kMode, kCta>::value;
+  using Cfg = PipeConfig<kCta, kAcc, kKA>;
   static_assert(kAcc == 1 || (kCta == 2 && (kMode == kModeDHidden || kMode == kModeDW)), "two accumulators: gradient modes, CTA pairs");
   constexpr int kBufs = 2 / kAcc;                          // tensor-memory buffers of kAcc accumulators
   constexpr int kUnitN = kBN * kAcc;                       // output columns per unit
@@ -180,7 +187,8 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   constexpr int kStagesT = Cfg::stages;
   constexpr int kBNcta = kBN / kCta;                       // rows of B that this CTA loads
   constexpr uint32_t kBBytesCta = kBNcta * kBK * 2;
-  constexpr uint32_t kStageBytesCta = kABytes + kAcc * kBBytesCta;
+  constexpr uint32_t kAtomBytesCta = kABytes + kAcc * kBBytesCta;
+  constexpr uint32_t kStageBytesCta = kKA * kAtomBytesCta;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[kStagesT];
   __shared__ __align__(8) uint64_t bar_empty[kStagesT];
@@ -229,7 +237,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   tc_fence_after_sync();
   const uint32_t tmem_base = tmem_base_slot;
 
-  const int k_blocks = (args.K + kBK - 1) / kBK;
+  const int k_blocks = (args.K + kBK * kKA - 1) / (kBK * kKA);
   const int n_units = (kMode == kModeStats) ? args.m_tiles * args.n_split : args.m_tiles * args.n_tiles;
 
   if (warp == 0) {
@@ -255,42 +263,48 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           const int b_row = args.b_mn0 + n_tile * kUnitN + cta_rank * kBNcta;   // + kBN per further accumulator
           for (int kb = 0; kb < k_blocks; ++kb) {
             if (!mbar_wait_bounded(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p, kWaitLimitCycles)) goto producer_drain;
-            const uint32_t sa = smem_base + stage * kStageBytesCta;
-            const uint32_t sb = sa + kABytes;
-            const int ka = args.a_k0 + kb * kBK, kbb = args.b_k0 + kb * kBK;
             const uint32_t full = full0 + stage * (uint32_t)sizeof(uint64_t);
             if (kPair) {
               // both CTAs' bytes are counted on the issuing CTA's barrier, which alone is armed
               if (cta_rank == 0) mbar_arrive_expect_tx(smem_u32(&bar_full[stage]), 2 * kStageBytesCta);
-              if (kAmn) {
-#pragma unroll
-                for (int j = 0; j < kBM / 64; ++j) tma_load_2d_pair(sa + j * kChunkBytes, &map_a, full, a_row + j * 64, ka);
-              } else {
-                tma_load_2d_pair(sa, &map_a, full, ka, a_row);
-              }
-#pragma unroll
-              for (int q = 0; q < kAcc; ++q) {
-                if (kBmn) {
-#pragma unroll
-                  for (int j = 0; j < kBNcta / 64; ++j)
-                    tma_load_2d_pair(sb + q * kBBytesCta + j * kChunkBytes, &map_b, full, b_row + q * kBN + j * 64, kbb);
-                } else {
-                  tma_load_2d_pair(sb + q * kBBytesCta, &map_b, full, kbb, b_row + q * kBN);
-                }
-              }
             } else {
               mbar_arrive_expect_tx(full, kStageBytesCta);
-              if (kAmn) {
+            }
 #pragma unroll
-                for (int j = 0; j < kBM / 64; ++j) tma_load_2d(sa + j * kChunkBytes, &map_a, full, a_row + j * 64, ka);
-              } else {
-                tma_load_2d(sa, &map_a, full, ka, a_row);
-              }
-              if (kBmn) {
+            for (int t = 0; t < kKA; ++t) {
+              const uint32_t sa = smem_base + stage * kStageBytesCta + t * kAtomBytesCta;
+              const uint32_t sb = sa + kABytes;
+              const int ka = args.a_k0 + (kb * kKA + t) * kBK, kbb = args.b_k0 + (kb * kKA + t) * kBK;
+              if (kPair) {
+                if (kAmn) {
 #pragma unroll
-                for (int j = 0; j < kBNcta / 64; ++j) tma_load_2d(sb + j * kChunkBytes, &map_b, full, b_row + j * 64, kbb);
+                  for (int j = 0; j < kBM / 64; ++j) tma_load_2d_pair(sa + j * kChunkBytes, &map_a, full, a_row + j * 64, ka);
+                } else {
+                  tma_load_2d_pair(sa, &map_a, full, ka, a_row);
+                }
+#pragma unroll
+                for (int q = 0; q < kAcc; ++q) {
+                  if (kBmn) {
+#pragma unroll
+                    for (int j = 0; j < kBNcta / 64; ++j)
+                      tma_load_2d_pair(sb + q * kBBytesCta + j * kChunkBytes, &map_b, full, b_row + q * kBN + j * 64, kbb);
+                  } else {
+                    tma_load_2d_pair(sb + q * kBBytesCta, &map_b, full, kbb, b_row + q * kBN);
+                  }
+                }
               } else {
-                tma_load_2d(sb, &map_b, full, kbb, b_row);
+                if (kAmn) {
+#pragma unroll
+                  for (int j = 0; j < kBM / 64; ++j) tma_load_2d(sa + j * kChunkBytes, &map_a, full, a_row + j * 64, ka);
+                } else {
+                  tma_load_2d(sa, &map_a, full, ka, a_row);
+                }
+                if (kBmn) {
+#pragma unroll
+                  for (int j = 0; j < kBNcta / 64; ++j) tma_load_2d(sb + j * kChunkBytes, &map_b, full, b_row + j * 64, kbb);
+                } else {
+                  tma_load_2d(sb, &map_b, full, kbb, b_row);
+                }
               }
             }
             ++issued;
@@ -332,6 +346,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       constexpr uint64_t a_step = (kAmn ? kUmmaK * 128 : kUmmaK * 2) >> 4;
       constexpr uint64_t b_step = (kBmn ? kUmmaK * 128 : kUmmaK * 2) >> 4;
       constexpr uint64_t stage_step = kStageBytesCta >> 4;
+      constexpr uint64_t atom_step = kAtomBytesCta >> 4;
       const uint64_t da_base = kAmn ? make_smem_desc(smem_base, kChunkBytes, 1024) : make_smem_desc(smem_base, 16, 1024);
       const uint64_t db_base = kBmn ? make_smem_desc(smem_base + kABytes, kChunkBytes, 1024)
                                     : make_smem_desc(smem_base + kABytes, 16, 1024);
@@ -355,12 +370,17 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const uint64_t da = da_base + stage * stage_step;
             const uint64_t db = db_base + stage * stage_step;
 #pragma unroll
-            for (int q = 0; q < kAcc; ++q) {
+            for (int t = 0; t < kKA; ++t) {
 #pragma unroll
-              for (int k = 0; k < kBK / kUmmaK; ++k) {
-                const uint64_t dbq = db + q * (uint64_t)(kBBytesCta >> 4) + k * b_step;
-                if (kPair) umma_bf16_pair(tmem_d + q * kBN, da + k * a_step, dbq, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-                else umma_bf16(tmem_d + q * kBN, da + k * a_step, dbq, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+              for (int q = 0; q < kAcc; ++q) {
+#pragma unroll
+                for (int k = 0; k < kBK / kUmmaK; ++k) {
+                  const uint64_t daq = da + t * atom_step + k * a_step;
+                  const uint64_t dbq = db + t * atom_step + q * (uint64_t)(kBBytesCta >> 4) + k * b_step;
+                  const uint32_t acc = (kb > 0 || t > 0 || k > 0) ? 1u : 0u;
+                  if (kPair) umma_bf16_pair(tmem_d + q * kBN, daq, dbq, idesc, acc);
+                  else umma_bf16(tmem_d + q * kBN, daq, dbq, idesc, acc);
+                }
               }
             }
             if (kPair) {
@@ -424,7 +444,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const uint32_t buf = acc_iter % kBufs;
         const uint32_t buf_phase = (acc_iter / kBufs) & 1u;
         const int col_base = n_tile * kUnitN;
-        if (!mbar_wait_bounded(smem_u32(&bar_tmem_full[buf]), buf_phase, abort_p, kWaitLimitCycles)) goto role_done;
+        if (!mbar_wait_bounded<true>(smem_u32(&bar_tmem_full[buf]), buf_phase, abort_p, kWaitLimitCycles)) goto role_done;
         tc_fence_after_sync();
         const uint32_t taddr = tmem_base + buf * kUnitN + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll 1
