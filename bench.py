@@ -29,6 +29,10 @@ from paper_2507_19766_b200 import synth  # noqa: E402
 
 METRIC = "fused loss fwd+bwd tokens/sec at H=2048,V=151936; % of B200 bf16 tensor peak"
 NOMINAL_BF16_TFLOPS = 2250.0
+# DRAM bytes (read + write) per launch of each tensor-core kernel at the full ultra workload, from the ncu
+# capture summarised in profiles/launch_list_ultra_full_size.md.  They describe the kernels as they were at
+# that capture: set an entry to None when its kernel changes, until the counters are taken again.
+NCU_TRAFFIC_BYTES = {"ultra": {"stats": 41.775e9, "dz": 10.912e9, "d_hidden": 15.102e9, "d_W": 16.625e9}}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -312,7 +316,8 @@ def main():
     peak = peaks["bf16_tflops_sustained"]
     roofline = {"bound": "tensor", "kernel": f"umma_kernel<{dom}>", "achieved": achieved, "peak": peak,
                 "unit": "TFLOP/s", "frac": achieved / peak,
-                "peak_kind": f"bf16 sustained, {peaks['source']}", "traffic": None,
+                "peak_kind": f"bf16 sustained, {peaks['source']}",
+                "traffic": (NCU_TRAFFIC_BYTES.get(wl.name, {}).get(dom) if args.tokens == 0 and args.panel == 0 else None),
                 "flops_per_launch": flops_kernel * args.steps / n_launch,
                 "avg_launch_ms": kinds[dom]["ms_total"] / n_launch, "per_kernel": kinds}
     exec_tflops = 8.0 * wl.T * wl.H * wl.V * world * args.steps / (ms_total * 1e-3) / 1e12
