@@ -186,6 +186,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="ultra", choices=list(synth.WORKLOADS))
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--compact-steps", type=int, default=5, help="steps of the run with active-row compaction (0 = skip)")
     ap.add_argument("--cpu-rows", type=int, default=768, help="rows of the CPU-baseline sample (0 = skip)")
     ap.add_argument("--ref-rows", type=int, default=256)
     ap.add_argument("--panel", type=int, default=0, help="backward panel tokens (0 = library default)")
@@ -267,6 +268,44 @@ def main():
     value = tokens / (ms_total * 1e-3)
     stats = out.stats_host()
 
+    # ---- the same step with the backward restricted to the tokens whose coefficient is non-zero
+    compacted = None
+    if args.compact_steps > 0 and wl.dtype == "bf16":
+        import dataclasses
+        gp_c = dataclasses.replace(gp, compact_rows=True)
+        ws_c = B.alloc_workspace(gp_c, dev)
+
+        def step_c():
+            B.token_loss_fwd(gp_c, b.hidden, b.W, b.targets, b.old_logp, b.segment_version, b.advantages,
+                             b.seq_offsets, out=out, workspace=ws_c)
+            B.token_loss_bwd(gp_c, b.hidden, b.W, b.targets, out.lse, out.grad_coef, d_hidden=d_hidden, d_W=d_W,
+                             workspace=ws_c)
+            if dist is not None:
+                dp.reduce_step_outputs(d_W, out.loss)
+
+        for _ in range(warmup):
+            step_c()
+        fence()
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record()
+        for _ in range(args.compact_steps):
+            step_c()
+        c1.record()
+        fence()
+        assert B.check_status(ws_c) == B.OK
+        cms = torch.tensor([c0.elapsed_time(c1)], dtype=torch.float64, device=dev)
+        if dist is not None:
+            dist.all_reduce(cms, op=dist.ReduceOp.MAX)
+        cms = float(cms.item())
+        t_act = stats["n_active"]
+        compacted = {"value": world * wl.T * args.compact_steps / (cms * 1e-3), "unit": "tokens/s",
+                     "ms_per_step": cms / args.compact_steps, "steps": args.compact_steps,
+                     "active_tokens": t_act, "active_fraction": t_act / wl.T,
+                     "executed_tflops_per_gpu": (2.0 * wl.T + 6.0 * t_act) * wl.H * wl.V * args.compact_steps
+                                                / (cms * 1e-3) / 1e12,
+                     "note": "backward contractions on tokens with a non-zero coefficient only; same results"}
+        del ws_c
+
     # ---- end to end through the host-buffer entry point
     e2e = None
     if args.e2e_steps > 0:
@@ -334,7 +373,7 @@ def main():
                         "of_nominal_2250": exec_tflops / world / NOMINAL_BF16_TFLOPS, "peaks": peaks["source"]},
         "loss": stats["loss"], "mean_entropy": stats["mean_entropy"], "n_masked": stats["n_masked"],
         "n_active": stats["n_active"],
-        "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+        "roofline": roofline, "compacted": compacted, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
     }
     if world == 1 and args.cpu_rows > 0:
         line["cpu_baseline"] = cpu_baseline(host_batch, args.cpu_rows)

@@ -74,6 +74,11 @@ typedef struct {
   int32_t dw_accumulate;       /* bwd: 0 overwrite d_W, 1 add into it (micro-batching)                           */
   int32_t kernel_path;         /* ulorl_kernel_path_t; AUTO = tensor-core path for bf16, SIMT path for f32       */
   int32_t bwd_panel_tokens;    /* bwd: tokens per staging panel; 0 = library default                             */
+  int32_t compact_rows;        /* bwd, tensor path: 1 = run the three contractions only on tokens whose          */
+                               /* grad_coef is non-zero (masked, clipped and zero-advantage tokens add nothing   */
+                               /* to either gradient, Eq. 10); results are the same, the workspace grows by two  */
+                               /* [T, H] copies.  0 = all rows.  Part of the workspace size: pass the same value */
+                               /* to ulorl_workspace_bytes and to both calls.                                    */
 } ulorl_params_t;
 
 typedef struct {

@@ -44,6 +44,7 @@ class CParams(ctypes.Structure):
         ("entropy_target", ctypes.c_float), ("inv_temperature", ctypes.c_float),
         ("norm_tokens", ctypes.c_int64), ("current_version", ctypes.c_int32),
         ("dw_accumulate", ctypes.c_int32), ("kernel_path", ctypes.c_int32), ("bwd_panel_tokens", ctypes.c_int32),
+        ("compact_rows", ctypes.c_int32),
     ]
 
 
@@ -137,13 +138,14 @@ class Params:
     dw_accumulate: bool = False
     kernel_path: str = "auto"
     bwd_panel_tokens: int = 0
+    compact_rows: bool = False
 
     def to_c(self) -> CParams:
         return CParams(self.T, self.H, self.V, self.num_seqs, BF16 if self.dtype == "bf16" else F32,
                        _IS[self.is_mode], _MPT[self.mpt_mode], _ENT[self.ent_scope], int(self.adv_per_token),
                        self.clip_eps_low, self.clip_eps_high, self.mpt_tau, self.entropy_target,
                        self.inv_temperature, self.norm_tokens, self.current_version, int(self.dw_accumulate),
-                       _PATH[self.kernel_path], self.bwd_panel_tokens)
+                       _PATH[self.kernel_path], self.bwd_panel_tokens, int(self.compact_rows))
 
 
 def workspace_bytes(p: Params) -> int:

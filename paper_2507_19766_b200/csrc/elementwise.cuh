@@ -248,4 +248,114 @@ __global__ void finalize_kernel(int T, int n_blocks, double inv_N, const DecideP
   }
 }
 
+// ------------------------------------------------------------------------------------------
+// Active-row compaction of the backward.  Tokens whose d loss / d logp is exactly zero (masked
+// well-mastered positive tokens of Eq. 10, clipped tokens, zero advantage) add nothing to dHidden or
+// dW, so the backward contractions run on the remaining rows only.
+//   compact_count_kernel   active tokens per block of 256
+//   compact_offsets_kernel exclusive scan of the block counts (one block), total -> n_active
+//   compact_gather_kernel  position of every token among the active ones; hidden rows, targets, lse
+//                          and coefficient of the active tokens gathered in token order; the rows up
+//                          to the next multiple of 256 zero-filled (they are read as padding)
+//   compact_scatter_kernel dHidden rows back to their tokens, zeros for the inactive ones
+// ------------------------------------------------------------------------------------------
+constexpr int kCompactThreads = 256;
+
+__global__ void compact_count_kernel(int T, const float* __restrict__ grad_coef, int* __restrict__ block_count) {
+  const int t = blockIdx.x * kCompactThreads + threadIdx.x;
+  const int active = (t < T && grad_coef[t] != 0.f) ? 1 : 0;
+  const int n = __syncthreads_count(active);
+  if (threadIdx.x == 0) block_count[blockIdx.x] = n;
+}
+
+__global__ void compact_offsets_kernel(int n_blocks, const int* __restrict__ block_count, int* __restrict__ block_offset,
+                                       int* __restrict__ n_active) {
+  __shared__ int sh[1024];
+  // n_blocks can exceed the block size: every thread owns a contiguous run of blocks
+  const int per = (n_blocks + 1023) / 1024;
+  const int b0 = threadIdx.x * per, b1 = min(n_blocks, b0 + per);
+  int sum = 0;
+  for (int b = b0; b < b1; ++b) sum += block_count[b];
+  sh[threadIdx.x] = sum;
+  __syncthreads();
+  for (int off = 1; off < 1024; off <<= 1) {          // inclusive scan of the per-thread sums
+    const int v = threadIdx.x >= off ? sh[threadIdx.x - off] : 0;
+    __syncthreads();
+    sh[threadIdx.x] += v;
+    __syncthreads();
+  }
+  int run = sh[threadIdx.x] - sum;
+  for (int b = b0; b < b1; ++b) {
+    block_offset[b] = run;
+    run += block_count[b];
+  }
+  if (threadIdx.x == 1023) *n_active = sh[1023];
+}
+
+template <typename TIn>
+__global__ void compact_gather_kernel(int T, int H, const float* __restrict__ grad_coef, const int* __restrict__ block_offset,
+                                      const int* __restrict__ n_active, const TIn* __restrict__ hidden,
+                                      const int* __restrict__ targets, const float* __restrict__ lse,
+                                      int* __restrict__ position, TIn* __restrict__ hidden_c, int* __restrict__ targets_c,
+                                      float* __restrict__ lse_c, float* __restrict__ coef_c) {
+  __shared__ int sh_pos[kCompactThreads];
+  const int t = blockIdx.x * kCompactThreads + threadIdx.x;
+  const bool active = t < T && grad_coef[t] != 0.f;
+  // rank inside the block by warp ballots
+  const unsigned ballot = __ballot_sync(0xffffffffu, active);
+  __shared__ int warp_base[kCompactThreads / 32];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) warp_base[warp] = __popc(ballot);
+  __syncthreads();
+  int base = block_offset[blockIdx.x];
+  for (int w = 0; w < warp; ++w) base += warp_base[w];
+  const int pos = active ? base + __popc(ballot & ((1u << lane) - 1u)) : -1;
+  sh_pos[threadIdx.x] = pos;
+  if (t < T) position[t] = pos;
+  if (active) {
+    targets_c[pos] = targets[t];
+    lse_c[pos] = lse[t];
+    coef_c[pos] = grad_coef[t];
+  }
+  __syncthreads();
+  // rows: 16-byte vectors, the whole block cooperates on each active token of the block
+  const int vec_per_row = H * (int)sizeof(TIn) / 16;
+  for (int r = 0; r < kCompactThreads; ++r) {
+    const int p = sh_pos[r];
+    if (p < 0) continue;
+    const uint4* src = reinterpret_cast<const uint4*>(hidden + (size_t)(blockIdx.x * kCompactThreads + r) * H);
+    uint4* dst = reinterpret_cast<uint4*>(hidden_c + (size_t)p * H);
+    for (int v = threadIdx.x; v < vec_per_row; v += kCompactThreads) dst[v] = src[v];
+  }
+  // the last block zero-fills the padding rows [n_active, next multiple of 256)
+  if (blockIdx.x == gridDim.x - 1) {
+    const int n = *n_active;
+    const int n_pad = (n + 255) / 256 * 256;
+    for (int p = n; p < n_pad; ++p) {
+      uint4* dst = reinterpret_cast<uint4*>(hidden_c + (size_t)p * H);
+      for (int v = threadIdx.x; v < vec_per_row; v += kCompactThreads) dst[v] = make_uint4(0u, 0u, 0u, 0u);
+      if (threadIdx.x == 0) { targets_c[p] = 0; lse_c[p] = 0.f; coef_c[p] = 0.f; }
+    }
+  }
+}
+
+template <typename TIn>
+__global__ void compact_scatter_kernel(int T, int H, const int* __restrict__ position, const TIn* __restrict__ d_hidden_c,
+                                       TIn* __restrict__ d_hidden) {
+  // one block per 8 tokens, 16-byte vectors
+  const int vec_per_row = H * (int)sizeof(TIn) / 16;
+  for (int r = 0; r < 8; ++r) {
+    const int t = blockIdx.x * 8 + r;
+    if (t >= T) return;
+    const int p = position[t];
+    uint4* dst = reinterpret_cast<uint4*>(d_hidden + (size_t)t * H);
+    if (p >= 0) {
+      const uint4* src = reinterpret_cast<const uint4*>(d_hidden_c + (size_t)p * H);
+      for (int v = threadIdx.x; v < vec_per_row; v += blockDim.x) dst[v] = src[v];
+    } else {
+      for (int v = threadIdx.x; v < vec_per_row; v += blockDim.x) dst[v] = make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
+}
+
 }  // namespace ulorl

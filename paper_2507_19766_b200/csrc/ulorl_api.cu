@@ -40,6 +40,11 @@ struct Plan {
   int panel_tokens;
   size_t dz_ld;           // leading dimension of the dz panel (elements)
   size_t off_status, off_batch_mean, off_seq_sum, off_partials, off_acc_y, off_decide, off_dz, total;
+  bool compact;           // backward on the rows with a non-zero coefficient only (tensor path)
+  int compact_blocks;     // blocks of 256 tokens of the compaction kernels
+  size_t t_pad;           // rows of the compacted buffers
+  size_t off_n_active, off_blk_count, off_blk_offset, off_position, off_targets_c, off_lse_c, off_coef_c,
+      off_hidden_c, off_dh_c;
   int decide_blocks;
 };
 
@@ -62,6 +67,7 @@ static int validate_params(const ulorl_params_t* p) {
   if (!(p->clip_eps_low >= 0.f) || !(p->clip_eps_high >= 0.f) || p->clip_eps_low > 1.f) return ULORL_ERR_INVALID_ARG;
   if (!(p->mpt_tau > 0.f) || p->mpt_tau > 1.f) return ULORL_ERR_INVALID_ARG;
   if (p->norm_tokens < 0 || p->bwd_panel_tokens < 0) return ULORL_ERR_INVALID_ARG;
+  if (p->compact_rows != 0 && p->compact_rows != 1) return ULORL_ERR_INVALID_ARG;
   if (p->H % 8 != 0) return ULORL_ERR_UNSUPPORTED;
   return ULORL_OK;
 }
@@ -83,10 +89,11 @@ static Plan make_plan(const ulorl_params_t* p) {
   pl.n_split = (n_tiles + pl.tiles_per_split - 1) / pl.tiles_per_split;
   int panel = p->bwd_panel_tokens > 0 ? p->bwd_panel_tokens
                                       : (pl.tensor ? (cta_group() == 2 ? kDefaultPanelPair : kDefaultPanelTensor) : kDefaultPanelSimt);
-  panel = (panel + kBM - 1) / kBM * kBM;
-  const int t_round = (T + kBM - 1) / kBM * kBM;
+  const int panel_unit = pl.tensor ? kBM * cta_group() : kBM;   // whole row tiles: the dz kernel zero-fills to the tile end
+  panel = (panel + panel_unit - 1) / panel_unit * panel_unit;
+  const int t_round = (T + panel_unit - 1) / panel_unit * panel_unit;
   if (panel > t_round) panel = t_round;
-  if (panel < kBM) panel = kBM;
+  if (panel < panel_unit) panel = panel_unit;
   pl.panel_tokens = panel;
   pl.dz_ld = pl.tensor ? align_up((size_t)V, 64) : (size_t)V;
   pl.decide_blocks = (T + kDecideThreads - 1) / kDecideThreads;
@@ -98,6 +105,21 @@ static Plan make_plan(const ulorl_params_t* p) {
   pl.off_acc_y = off;       off = align_up(off + sizeof(float) * (size_t)(T > 0 ? T : 1), 256);
   pl.off_decide = off;      off = align_up(off + sizeof(DecidePartial) * (size_t)(pl.decide_blocks > 0 ? pl.decide_blocks : 1), 1024);
   pl.off_dz = off;          off = align_up(off + (size_t)panel * pl.dz_ld * (pl.tensor ? 2 : 4), 1024);
+  pl.compact = pl.tensor && p->compact_rows != 0;
+  pl.compact_blocks = (T + kCompactThreads - 1) / kCompactThreads;
+  pl.t_pad = align_up((size_t)(T > 0 ? T : 1), 256) + 256;
+  if (pl.compact) {
+    const size_t nb = (size_t)(pl.compact_blocks > 0 ? pl.compact_blocks : 1);
+    pl.off_n_active = off;   off += 256;
+    pl.off_blk_count = off;  off = align_up(off + 4 * nb, 256);
+    pl.off_blk_offset = off; off = align_up(off + 4 * nb, 256);
+    pl.off_position = off;   off = align_up(off + 4 * pl.t_pad, 256);
+    pl.off_targets_c = off;  off = align_up(off + 4 * pl.t_pad, 256);
+    pl.off_lse_c = off;      off = align_up(off + 4 * pl.t_pad, 256);
+    pl.off_coef_c = off;     off = align_up(off + 4 * pl.t_pad, 256);
+    pl.off_hidden_c = off;   off = align_up(off + 2 * pl.t_pad * (size_t)p->H, 1024);
+    pl.off_dh_c = off;       off = align_up(off + 2 * pl.t_pad * (size_t)p->H, 1024);
+  }
   pl.total = off;
   return pl;
 }
@@ -455,14 +477,46 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
   if (pl.tensor) {
     __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(ws + pl.off_dz);
     const int tile_m = kBM * cta_group();
+    // With compaction the three contractions run on gathered copies of the active rows; how many
+    // there are is only known on the device, so every launch is sized for the worst case and reads
+    // the count itself.
+    const int* n_active = nullptr;
+    void* d_hidden_out = d_hidden;
+    if (pl.compact) {
+      int* blk_count = reinterpret_cast<int*>(ws + pl.off_blk_count);
+      int* blk_offset = reinterpret_cast<int*>(ws + pl.off_blk_offset);
+      int* position = reinterpret_cast<int*>(ws + pl.off_position);
+      int* n_act = reinterpret_cast<int*>(ws + pl.off_n_active);
+      int* targets_c = reinterpret_cast<int*>(ws + pl.off_targets_c);
+      float* lse_c = reinterpret_cast<float*>(ws + pl.off_lse_c);
+      float* coef_c = reinterpret_cast<float*>(ws + pl.off_coef_c);
+      __nv_bfloat16* hidden_c = reinterpret_cast<__nv_bfloat16*>(ws + pl.off_hidden_c);
+      compact_count_kernel<<<pl.compact_blocks, kCompactThreads, 0, stream>>>(T, grad_coef, blk_count);
+      ULORL_LAUNCH_CHECK();
+      compact_offsets_kernel<<<1, 1024, 0, stream>>>(pl.compact_blocks, blk_count, blk_offset, n_act);
+      ULORL_LAUNCH_CHECK();
+      compact_gather_kernel<__nv_bfloat16><<<pl.compact_blocks, kCompactThreads, 0, stream>>>(
+          T, H, grad_coef, blk_offset, n_act, static_cast<const __nv_bfloat16*>(hidden), targets, lse, position,
+          hidden_c, targets_c, lse_c, coef_c);
+      ULORL_LAUNCH_CHECK();
+      if (!params->dw_accumulate && cudaMemsetAsync(d_W, 0, sizeof(float) * (size_t)V * H, stream) != cudaSuccess)
+        return ULORL_ERR_CUDA;
+      n_active = n_act;
+      hidden = hidden_c;
+      targets = targets_c;
+      lse = lse_c;
+      grad_coef = coef_c;
+      d_hidden_out = ws + pl.off_dh_c;
+    }
+    const uint64_t hidden_rows = pl.compact ? (uint64_t)pl.t_pad : (uint64_t)T;
     CUtensorMap map_hidden_k, map_w_k, map_w_mn, map_hidden_mn;
-    st = make_map_bf16(&map_hidden_k, hidden, (uint64_t)T, (uint64_t)H, (uint64_t)H, kBK, kBM);
+    st = make_map_bf16(&map_hidden_k, hidden, hidden_rows, (uint64_t)H, (uint64_t)H, kBK, kBM);
     if (st != ULORL_OK) return st;
     st = make_map_bf16(&map_w_k, W, (uint64_t)V, (uint64_t)H, (uint64_t)H, kBK, kBN / cta_group());
     if (st != ULORL_OK) return st;
     st = make_map_bf16(&map_w_mn, W, (uint64_t)V, (uint64_t)H, (uint64_t)H, 64, kBK);
     if (st != ULORL_OK) return st;
-    st = make_map_bf16(&map_hidden_mn, hidden, (uint64_t)T, (uint64_t)H, (uint64_t)H, 64, kBK);
+    st = make_map_bf16(&map_hidden_mn, hidden, hidden_rows, (uint64_t)H, (uint64_t)H, 64, kBK);
     if (st != ULORL_OK) return st;
     CUtensorMap map_dw_out;   // d_W as the target of 128-row x 32-column float tiles
     st = make_map(&map_dw_out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, d_W, (uint64_t)V, (uint64_t)H, (uint64_t)H, 32, kBM);
@@ -481,6 +535,7 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
         a.kappa = kappa;
         a.targets = targets; a.lse = lse; a.grad_coef = grad_coef; a.grad_loss = grad_loss;
         a.dz = dz; a.dz_ld = pl.dz_ld; a.dz_cols = (int)pl.dz_ld;
+        a.dyn_rows = n_active; a.dyn_base = t0;
         a.status = status;
         st = launch_umma<kModeDz>(map_hidden_k, map_w_k, map_w_k, a, stream);
         if (st != ULORL_OK) return st;
@@ -498,8 +553,9 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
         a.n_tiles = (H + grad_unit_cols() - 1) / grad_unit_cols();
         a.group_m = kGradRasterGroup;
         a.row0 = t0;
-        a.d_hidden = static_cast<__nv_bfloat16*>(d_hidden);
+        a.d_hidden = static_cast<__nv_bfloat16*>(d_hidden_out);
         a.out_ld = (size_t)H;
+        a.dyn_rows = n_active; a.dyn_base = t0;
         a.status = status;
         st = launch_umma<kModeDHidden>(map_dz_k, map_w_mn, map_w_mn, a, stream);
         if (st != ULORL_OK) return st;
@@ -514,11 +570,18 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
         a.b_k0 = t0;
         a.d_W = d_W;
         a.out_ld = (size_t)H;
-        a.accumulate = (panel > 0 || params->dw_accumulate) ? 1 : 0;
+        a.accumulate = (panel > 0 || params->dw_accumulate || pl.compact) ? 1 : 0;
+        a.dyn_rows = n_active; a.dyn_base = t0;
         a.status = status;
         st = launch_umma<kModeDW>(map_dz_mn, map_hidden_mn, map_dw_out, a, stream);
         if (st != ULORL_OK) return st;
       }
+    }
+    if (pl.compact) {
+      compact_scatter_kernel<__nv_bfloat16><<<(T + 7) / 8, 256, 0, stream>>>(
+          T, H, reinterpret_cast<const int*>(ws + pl.off_position),
+          reinterpret_cast<const __nv_bfloat16*>(ws + pl.off_dh_c), static_cast<__nv_bfloat16*>(d_hidden));
+      ULORL_LAUNCH_CHECK();
     }
     return ULORL_OK;
   }

@@ -83,6 +83,8 @@ struct UmmaArgs {
   size_t out_ld;
   int accumulate;
   int* status;
+  const int* dyn_rows;      // optional device count of rows of the whole (compacted) batch: the launch then
+  int dyn_base;             // covers rows [dyn_base, min(dyn_base + capacity, *dyn_rows)) of it (M, or K for d_W)
 };
 
 template <int kMode>
@@ -174,8 +176,22 @@ __device__ __forceinline__ void dz_chunk(const uint32_t (&raw)[32], int nvalid, 
 template <int kMode, int kCta, int kAcc>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-            const __grid_constant__ CUtensorMap map_c, const UmmaArgs args) {
+            const __grid_constant__ CUtensorMap map_c, const UmmaArgs args_in) {
   using namespace ptx;
+  UmmaArgs args = args_in;
+  if (args.dyn_rows != nullptr) {
+    // The number of rows is only known on the device (rows kept by the compaction of the backward):
+    // this launch was sized for its capacity and shrinks itself to what is really there.
+    int n = *args.dyn_rows - args.dyn_base;
+    if (kMode == kModeDW) {
+      n = n < 0 ? 0 : (n > args.K ? args.K : n);
+      args.K = n;
+    } else {
+      n = n < 0 ? 0 : (n > args.M ? args.M : n);
+      args.M = n;
+      args.m_tiles = (n + kBM * kCta - 1) / (kBM * kCta);
+    }
+  }
   constexpr int kKA = KAtoms<kMode, kCta>::value;
   using Cfg = PipeConfig<kCta, kAcc, kKA>;
   static_assert(kAcc == 1 || (kCta == 2 && (kMode == kModeDHidden || kMode == kModeDW)), "two accumulators: gradient modes, CTA pairs");
@@ -238,7 +254,8 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   const uint32_t tmem_base = tmem_base_slot;
 
   const int k_blocks = (args.K + kBK * kKA - 1) / (kBK * kKA);
-  const int n_units = (kMode == kModeStats) ? args.m_tiles * args.n_split : args.m_tiles * args.n_tiles;
+  const int n_units = (k_blocks == 0) ? 0
+                      : (kMode == kModeStats) ? args.m_tiles * args.n_split : args.m_tiles * args.n_tiles;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (every CTA)
@@ -470,7 +487,11 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             uint32_t packed[16];
             if (nvalid >= 32) dz_chunk<true>(raw, 32, y - col0, coef, c2, lse2, packed);
             else dz_chunk<false>(raw, nvalid, y - col0, coef, c2, lse2, packed);
-            if (row_ok) {
+            if (!row_ok) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) packed[j] = 0u;   // rows past M of a written tile read as zero later
+            }
+            {
               uint4* dst = reinterpret_cast<uint4*>(args.dz + (size_t)row * args.dz_ld + col0);
               const int ncols = min(32, args.dz_cols - col0);     // multiple of 8
 #pragma unroll

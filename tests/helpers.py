@@ -20,7 +20,7 @@ def both_params(batch: synth.Batch, **over):
               clip_eps_high=wl.clip_eps_high, mpt_tau=wl.mpt_tau, entropy_target=wl.entropy_target,
               inv_temperature=1.0, norm_tokens=0, current_version=batch.current_version)
     extra = {k: over.pop(k) for k in list(over) if k in ("kernel_path", "bwd_panel_tokens", "dw_accumulate",
-                                                         "adv_per_token")}
+                                                         "adv_per_token", "compact_rows")}
     kw.update(over)
     gp = Params(T=wl.T, H=wl.H, V=wl.V, num_seqs=wl.S, dtype=wl.dtype, **kw, **extra)
     op = O.OracleParams(**kw)

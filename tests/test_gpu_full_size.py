@@ -119,6 +119,19 @@ def test_full_size_workload_against_sampled_oracle(name):
     torch.cuda.synchronize()
     assert rel_l2(dW2.cpu().numpy(), dW_host.numpy()) <= 1e-4       # same sum, other panel boundaries
     del dW2, ws2
+    # the compacted backward (rows with a zero coefficient dropped) gives the same gradients
+    gp3, _ = both_params(batch, compact_rows=True)
+    ws3c = B.alloc_workspace(gp3, DEV)
+    dH3, dW3 = B.token_loss_bwd(gp3, b.hidden, b.W, b.targets, out.lse, out.grad_coef, workspace=ws3c)
+    torch.cuda.synchronize()
+    assert B.check_status(ws3c) == B.OK
+    assert rel_l2(dW3.cpu().numpy(), dW_host.numpy()) <= 1e-4
+    ta_all = torch.from_numpy(rows).to(DEV)
+    assert rel_l2(dH3[ta_all].float().cpu().numpy()[sel], dH_ref) <= TOL_GRAD
+    zero_rows = np.nonzero(g == 0)[0][:4096]
+    if zero_rows.size:
+        assert float(dH3[torch.from_numpy(zero_rows).to(DEV)].float().abs().max()) == 0.0
+    del dH3, dW3, ws3c
 
     # ---- dW: sub-batch of the sampled active rows against the full oracle, same N and same g
     n_sub = int(active.size)

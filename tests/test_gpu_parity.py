@@ -321,3 +321,50 @@ def test_repeated_runs_are_bit_identical():
     b = gpu_fwd_bwd(batch, gp)
     assert torch.equal(a[0].logp, b[0].logp) and torch.equal(a[0].loss, b[0].loss)
     assert torch.equal(a[1], b[1]) and torch.equal(a[2], b[2])
+
+
+# --------------------------------------------------------------------------- active-row compaction
+@pytest.mark.parametrize("panel", [0, 256])
+def test_compacted_backward_matches_dense_and_oracle(panel):
+    """Rows with a zero coefficient (masked, clipped, zero advantage) are dropped from the backward
+    contractions; the gradients must not change."""
+    wl = synth.WORKLOADS["small"].scaled(T=1500, S=6, H=256, V=3000, lengths="lognormal:200:500", segment_len=64,
+                                         planted=0.5, beta_planted=(100.0, 220.0), mpt_mode="always",
+                                         noise="const:0.15", adv="bern:0.5:3")
+    batch = synth.make_batch(wl, seed=33)
+    gp_d, op = both_params(batch, bwd_panel_tokens=panel)
+    gp_c, _ = both_params(batch, bwd_panel_tokens=panel, compact_rows=True)
+    out_d, dH_d, dW_d = gpu_fwd_bwd(batch, gp_d)
+    out_c, dH_c, dW_c = gpu_fwd_bwd(batch, gp_c)
+    st = out_c.stats_host()
+    assert 0 < st["n_active"] < wl.T - 100 and st["n_masked"] > 20 and st["n_clip_high"] + st["n_clip_low"] > 0
+    assert torch.equal(out_d.grad_coef, out_c.grad_coef)
+    assert torch.equal(dH_d, dH_c)                       # a row's reduction over V does not depend on its position
+    assert rel_l2(dW_c.cpu().numpy(), dW_d.cpu().numpy()) <= 1e-5
+    inactive = (out_c.grad_coef == 0)
+    assert float(dH_c[inactive].float().abs().max()) == 0.0
+    check_against_oracle(batch, gp_c, op)
+
+
+def test_compacted_backward_with_nothing_active_and_with_accumulation():
+    wl = synth.WORKLOADS["small"].scaled(T=300, S=2, H=128, V=1024, lengths="tiny", planted=1.0,
+                                         beta_planted=(400.0, 500.0), adv="plus1", mpt_mode="always")
+    batch = synth.make_batch(wl, seed=6)
+    gp, _ = both_params(batch, compact_rows=True)
+    out, dH, dW = gpu_fwd_bwd(batch, gp)
+    assert out.stats_host()["n_active"] == 0
+    assert float(dH.float().abs().max()) == 0.0 and float(dW.abs().max()) == 0.0
+    # accumulation into a caller's d_W
+    wl2 = synth.WORKLOADS["small"].scaled(T=600, S=3, H=128, V=1500, lengths="tiny", planted=0.4,
+                                          beta_planted=(300.0, 500.0), mpt_mode="always")
+    b2 = synth.make_batch(wl2, seed=14)
+    gp_d, _ = both_params(b2)
+    gp_a, _ = both_params(b2, compact_rows=True, dw_accumulate=True)
+    _, _, dW_ref = gpu_fwd_bwd(b2, gp_d)
+    b = b2.to(DEV)
+    ws = B.alloc_workspace(gp_a, DEV)
+    out = B.token_loss_fwd(gp_a, b.hidden, b.W, b.targets, b.old_logp, b.segment_version, b.advantages, b.seq_offsets,
+                           workspace=ws)
+    dW = torch.ones(wl2.V, wl2.H, dtype=torch.float32, device=DEV)
+    B.token_loss_bwd(gp_a, b.hidden, b.W, b.targets, out.lse, out.grad_coef, d_W=dW, workspace=ws)
+    assert rel_l2((dW - 1.0).cpu().numpy(), dW_ref.cpu().numpy()) <= 1e-4
