@@ -350,15 +350,23 @@ def main():
                  "tflops": (flops_kernel * args.steps / (v[0] * 1e-3) / 1e12) if v[0] > 0 else None}
              for k, v in kt.items()}
     dom = max(kinds, key=lambda k: kinds[k]["ms_total"])
-    n_launch = max(kinds[dom]["launches"], 1)
-    achieved = flops_kernel * args.steps / n_launch / (kinds[dom]["ms_total"] / n_launch * 1e-3) / 1e12
-    peak = peaks["bf16_tflops_sustained"]
-    roofline = {"bound": "tensor", "kernel": f"umma_kernel<{dom}>", "achieved": achieved, "peak": peak,
-                "unit": "TFLOP/s", "frac": achieved / peak,
-                "peak_kind": f"bf16 sustained, {peaks['source']}",
-                "traffic": (NCU_TRAFFIC_BYTES.get(wl.name, {}).get(dom) if args.tokens == 0 and args.panel == 0 else None),
-                "flops_per_launch": flops_kernel * args.steps / n_launch,
-                "avg_launch_ms": kinds[dom]["ms_total"] / n_launch, "per_kernel": kinds}
+    if kinds[dom]["ms_total"] > 0:
+        n_launch = max(kinds[dom]["launches"], 1)
+        achieved = flops_kernel * args.steps / n_launch / (kinds[dom]["ms_total"] / n_launch * 1e-3) / 1e12
+        peak = peaks["bf16_tflops_sustained"]
+        roofline = {"bound": "tensor", "kernel": f"umma_kernel<{dom}>", "achieved": achieved, "peak": peak,
+                    "unit": "TFLOP/s", "frac": achieved / peak,
+                    "peak_kind": f"bf16 sustained, {peaks['source']}",
+                    "traffic": (NCU_TRAFFIC_BYTES.get(wl.name, {}).get(dom)
+                                if args.tokens == 0 and args.panel == 0 else None),
+                    "flops_per_launch": flops_kernel * args.steps / n_launch,
+                    "avg_launch_ms": kinds[dom]["ms_total"] / n_launch, "per_kernel": kinds}
+    else:   # float32 workloads run on the CUDA-core kernels, which the per-kernel timer does not bracket
+        achieved = 8.0 * wl.T * wl.H * wl.V * args.steps / (ms_total * 1e-3) / 1e12
+        roofline = {"bound": "alu", "kernel": "simt kernels (whole step)", "achieved": achieved,
+                    "peak": 148 * 128 * 2 * 1.965e9 / 1e12, "unit": "TFLOP/s",
+                    "frac": achieved / (148 * 128 * 2 * 1.965e9 / 1e12),
+                    "peak_kind": "fp32 FMA: 148 SMs x 128 lanes x 2 flop x 1.965 GHz", "traffic": None}
     exec_tflops = 8.0 * wl.T * wl.H * wl.V * world * args.steps / (ms_total * 1e-3) / 1e12
     line = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": warmup,

@@ -64,7 +64,7 @@ WORKLOADS = {
     "qwen": Workload("qwen", 2, T=65536, S=32, H=2048, V=151936, dtype="bf16",
                      lengths="longtail:1024:32768", segment_len=8192, max_segments=4,
                      noise="const:0.1", adv="bern:0.3:16", planted=0.4, sampled=0.0,
-                     mpt_mode="dynamic"),
+                     mpt_mode="always"),      # static masking (Section 3.2.1), so that the planted rows are masked
     "mixed": Workload("mixed", 3, T=262144, S=64, H=2048, V=151936, dtype="bf16",
                       lengths="pareto:1.2:131072", segment_len=16384, max_segments=8,
                       noise="stale:0.02", adv="bern:0.3:16", planted=0.4, sampled=0.0,

@@ -87,6 +87,8 @@ def test_full_size_workload_against_sampled_oracle(name):
         assert seq_ent[0] < wl.entropy_target and st["n_masked"] > wl.T // 2 and st["n_active"] > wl.T // 20
     if name == "mixed":
         assert st["n_clip_high"] == 0 and st["n_clip_low"] == 0
+    if name == "qwen":         # static masking: planted targets of positive sequences are masked
+        assert st["n_mpt"] > 0 and st["n_masked"] == st["n_mpt"]
 
     # ---- sampled rows of dHidden (rows are independent given g_t)
     active = rows[g[rows] != 0]
