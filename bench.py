@@ -148,7 +148,7 @@ def run_reference(args):
         return
     wl_full = synth.WORKLOADS[args.workload]
     n_rows = args.ref_rows
-    wl = wl_full.scaled(T=n_rows * args.steps if False else n_rows, S=1, lengths="single",
+    wl = wl_full.scaled(T=n_rows, S=1, lengths="single",
                         segment_len=max(1, n_rows // wl_full.max_segments))
     dev = "cuda" if torch.cuda.is_available() else "cpu"
     batch = synth.make_batch(wl, device=dev)

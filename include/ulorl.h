@@ -177,8 +177,9 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params,
                          void* d_hidden, float* d_W,
                          void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* Synchronises the stream, reads the workspace status word and returns it (ULORL_OK, or
- * ULORL_ERR_DEVICE_TIMEOUT / ULORL_ERR_BAD_TARGET / ULORL_ERR_CUDA). */
+/* Synchronises the stream, reads the workspace status word and returns it: ULORL_OK, or
+ * ULORL_ERR_DEVICE_TIMEOUT, ULORL_ERR_INVALID_ARG (seq_offsets on the device were not
+ * 0 = o[0] <= ... <= o[S] = T; the offending ranges were clamped), ULORL_ERR_BAD_TARGET, ULORL_ERR_CUDA. */
 int ulorl_check_status(void* workspace, void* cuda_stream);
 
 const char* ulorl_status_string(int status);

@@ -15,6 +15,7 @@ constexpr int kMaxSplits = 32;
 // Device status word (first int of the workspace).  Bits, so that several problems can be kept.
 constexpr int kStatusTimeout = 1;
 constexpr int kStatusBadTarget = 2;
+constexpr int kStatusBadOffsets = 4;   // seq_offsets not 0 = o[0] <= o[1] <= ... <= o[S] = T
 
 // Per-block partial results of the decision kernel, reduced in block order by a final kernel
 // so that the loss and the statistics do not depend on scheduling.

@@ -41,11 +41,18 @@ __global__ void merge_splits_kernel(int T, int n_split, float kappa, const float
 // ------------------------------------------------------------------------------------------
 constexpr int kSeqThreads = 256;
 
-__global__ void seq_entropy_kernel(int S, const int* __restrict__ seq_offsets, const float* __restrict__ entropy,
-                                   double* __restrict__ seq_sum, float* __restrict__ seq_entropy) {
+__global__ void seq_entropy_kernel(int S, int T, const int* __restrict__ seq_offsets, const float* __restrict__ entropy,
+                                   double* __restrict__ seq_sum, float* __restrict__ seq_entropy, int* __restrict__ status) {
   __shared__ double red[kSeqThreads];
   const int i = blockIdx.x;
-  const int a = seq_offsets[i], b = seq_offsets[i + 1];
+  int a = seq_offsets[i], b = seq_offsets[i + 1];
+  // offsets are device data the host never saw: a bad pair is reported and clamped, never followed out of range
+  const bool bad = a < 0 || b < a || b > T || (i == 0 && a != 0) || (i == S - 1 && b != T);
+  if (bad) {
+    if (threadIdx.x == 0) atomicOr(status, kStatusBadOffsets);
+    a = a < 0 ? 0 : (a > T ? T : a);
+    b = b < a ? a : (b > T ? T : b);
+  }
   double acc = 0.0;
   for (int t = a + threadIdx.x; t < b; t += kSeqThreads) acc += (double)entropy[t];
   red[threadIdx.x] = acc;

@@ -297,7 +297,7 @@ static int run_decide(const ulorl_params_t* p, const Plan& pl, const float* logp
   DecidePartial* partials = reinterpret_cast<DecidePartial*>(ws + pl.off_decide);
   // the gate needs a float array of per-sequence means even when the caller does not want it back
   float* seq_ent_out = seq_entropy;
-  seq_entropy_kernel<<<S, kSeqThreads, 0, stream>>>(S, seq_offsets, entropy, seq_sum, seq_ent_out);
+  seq_entropy_kernel<<<S, kSeqThreads, 0, stream>>>(S, T, seq_offsets, entropy, seq_sum, seq_ent_out, status);
   ULORL_LAUNCH_CHECK();
   batch_entropy_kernel<<<1, 32, 0, stream>>>(S, T, seq_sum, batch_mean);
   ULORL_LAUNCH_CHECK();
@@ -367,6 +367,7 @@ int ulorl_check_status(void* workspace, void* cuda_stream) {
   if (cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return ULORL_ERR_CUDA;
   if (cudaStreamSynchronize(stream) != cudaSuccess) return ULORL_ERR_CUDA;
   if (word & kStatusTimeout) return ULORL_ERR_DEVICE_TIMEOUT;
+  if (word & kStatusBadOffsets) return ULORL_ERR_INVALID_ARG;
   if (word & kStatusBadTarget) return ULORL_ERR_BAD_TARGET;
   return ULORL_OK;
 }

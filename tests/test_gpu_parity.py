@@ -368,3 +368,69 @@ def test_compacted_backward_with_nothing_active_and_with_accumulation():
     dW = torch.ones(wl2.V, wl2.H, dtype=torch.float32, device=DEV)
     B.token_loss_bwd(gp_a, b.hidden, b.W, b.targets, out.lse, out.grad_coef, d_W=dW, workspace=ws)
     assert rel_l2((dW - 1.0).cpu().numpy(), dW_ref.cpu().numpy()) <= 1e-4
+
+
+# --------------------------------------------------------------------------- host-buffer step, timing aid, bad offsets
+def test_host_buffer_step_matches_device_calls():
+    wl = synth.WORKLOADS["small"].scaled(T=900, S=4, H=256, V=2500, lengths="tiny", planted=0.3,
+                                         beta_planted=(100.0, 200.0), mpt_mode="always")
+    batch = synth.make_batch(wl, seed=41)
+    gp, _ = both_params(batch)
+    out, dH, dW = gpu_fwd_bwd(batch, gp)
+    arena = torch.empty(B.host_step_arena_bytes(gp), dtype=torch.uint8, device=DEV)
+    pin = lambda t: t.contiguous().pin_memory()
+    ho = dict(logp=torch.empty(wl.T).pin_memory(), entropy=torch.empty(wl.T).pin_memory(),
+              flags=torch.empty(wl.T, dtype=torch.uint8).pin_memory(), seq_entropy=torch.empty(wl.S).pin_memory(),
+              loss=torch.empty(1).pin_memory(), stats=torch.empty(out.stats.numel(), dtype=torch.uint8).pin_memory(),
+              d_hidden=torch.empty(wl.T, wl.H, dtype=torch.bfloat16).pin_memory(),
+              d_W=torch.empty(wl.V, wl.H).pin_memory())
+    for _ in range(2):                                   # the arena is reusable across calls
+        B.token_loss_step_host(gp, arena, pin(batch.hidden), pin(batch.W), pin(batch.targets), pin(batch.old_logp),
+                               pin(batch.segment_version), pin(batch.advantages), pin(batch.seq_offsets), **ho)
+        torch.cuda.synchronize()
+    assert torch.equal(ho["logp"], out.logp.cpu()) and torch.equal(ho["entropy"], out.entropy.cpu())
+    assert torch.equal(ho["flags"], out.flags.cpu()) and torch.equal(ho["loss"], out.loss.cpu())
+    assert torch.equal(ho["d_hidden"], dH.cpu()) and torch.equal(ho["d_W"], dW.cpu())
+    assert B.decode_stats(ho["stats"]) == out.stats_host()
+    with pytest.raises(B.UlorlError, match="workspace"):
+        B.token_loss_step_host(gp, arena[:1024], pin(batch.hidden), pin(batch.W), pin(batch.targets),
+                               pin(batch.old_logp), pin(batch.segment_version), pin(batch.advantages),
+                               pin(batch.seq_offsets), **ho)
+
+
+def test_kernel_timing_counts_the_tensor_core_launches():
+    wl = synth.WORKLOADS["small"].scaled(T=700, S=2, H=256, V=2048, lengths="tiny")
+    batch = synth.make_batch(wl, seed=43)
+    gp, _ = both_params(batch, bwd_panel_tokens=256)
+    n0 = B.launch_count()
+    B.kernel_timing_begin()
+    gpu_fwd_bwd(batch, gp)
+    kt = B.kernel_timing_end()
+    panels = -(-wl.T // B_panel_rows(gp))
+    assert kt["stats"][1] == 1 and kt["dz"][1] == panels and kt["d_hidden"][1] == panels and kt["d_W"][1] == panels
+    assert all(ms > 0 for ms, n in kt.values())
+    assert B.launch_count() - n0 == 1 + 1 + 4 + 3 * panels      # stats, merge, decision stage (4), three per panel
+
+
+def B_panel_rows(gp):
+    # panels are whole row tiles of the kernels in use (256 tokens for CTA pairs, 128 otherwise)
+    import os
+    unit = 128 if os.environ.get("ULORL_CTA_GROUP", "2").startswith("1") else 256
+    return -(-gp.bwd_panel_tokens // unit) * unit
+
+
+def test_inconsistent_sequence_offsets_are_reported_not_followed():
+    wl = synth.WORKLOADS["small"].scaled(T=300, S=3, H=64, V=512, lengths="tiny")
+    batch = synth.make_batch(wl, seed=45)
+    gp, _ = both_params(batch)
+    b = batch.to(DEV)
+    ws = B.alloc_workspace(gp, DEV)
+    bad = b.seq_offsets.clone()
+    bad[2] = 5000                                        # beyond T
+    out = B.token_loss_fwd(gp, b.hidden, b.W, b.targets, b.old_logp, b.segment_version, b.advantages, bad,
+                           workspace=ws)
+    assert B.check_status(ws) == -1
+    assert torch.isfinite(out.seq_entropy).all()
+    out = B.token_loss_fwd(gp, b.hidden, b.W, b.targets, b.old_logp, b.segment_version, b.advantages, b.seq_offsets,
+                           workspace=ws)
+    assert B.check_status(ws) == B.OK
