@@ -187,7 +187,7 @@ def main():
     ap.add_argument("--workload", default="ultra", choices=list(synth.WORKLOADS))
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--compact-steps", type=int, default=5, help="steps of the run with active-row compaction (0 = skip)")
-    ap.add_argument("--cpu-rows", type=int, default=768, help="rows of the CPU-baseline sample (0 = skip)")
+    ap.add_argument("--cpu-rows", type=int, default=2048, help="rows of the CPU-baseline sample (0 = skip)")
     ap.add_argument("--ref-rows", type=int, default=256)
     ap.add_argument("--panel", type=int, default=0, help="backward panel tokens (0 = library default)")
     ap.add_argument("--tokens", type=int, default=0,
