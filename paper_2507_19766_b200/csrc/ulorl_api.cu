@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <functional>
 #include <vector>
 
 #include "common.cuh"
@@ -333,6 +334,15 @@ static int empty_forward(void* workspace, size_t workspace_bytes, float* loss, v
   return ULORL_OK;
 }
 
+// Points at which the host-buffer step interleaves its copies with the two passes.  The forward
+// launches the statistics kernel once per chunk of tokens (all at once without hooks), the backward
+// reports every token panel whose d_hidden rows are final.
+struct StepHooks {
+  int chunk_tokens = 0;
+  std::function<int(int, int)> before_stats_chunk;    // (first token, tokens) -> status
+  std::function<int(int, int)> after_dhidden_panel;   // (first token, tokens) -> status; dense backward only
+};
+
 }  // namespace ulorl
 
 using namespace ulorl;
@@ -392,11 +402,11 @@ int ulorl_token_loss_decide(const ulorl_params_t* params, const float* logp, con
                     grad_coef, flags, seq_entropy, loss, stats, ws, stream);
 }
 
-int ulorl_token_loss_fwd(const ulorl_params_t* params, const void* hidden, const void* W, const int32_t* targets,
-                         const float* old_logp, const int32_t* segment_version, const float* advantages,
-                         const int32_t* seq_offsets, const float* entropy_supplied, float* logp, float* entropy,
-                         float* lse, float* grad_coef, uint8_t* flags, float* seq_entropy, float* loss, void* stats,
-                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+static int fwd_impl(const ulorl_params_t* params, const void* hidden, const void* W, const int32_t* targets,
+                    const float* old_logp, const int32_t* segment_version, const float* advantages,
+                    const int32_t* seq_offsets, const float* entropy_supplied, float* logp, float* entropy,
+                    float* lse, float* grad_coef, uint8_t* flags, float* seq_entropy, float* loss, void* stats,
+                    void* workspace, size_t workspace_bytes, void* cuda_stream, const StepHooks* hooks) {
   int st = validate_params(params);
   if (st != ULORL_OK) return st;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
@@ -421,21 +431,37 @@ int ulorl_token_loss_fwd(const ulorl_params_t* params, const void* hidden, const
     if (st != ULORL_OK) return st;
     st = make_map_bf16(&map_b, W, (uint64_t)V, (uint64_t)H, (uint64_t)H, kBK, kBN / cta_group());
     if (st != ULORL_OK) return st;
-    UmmaArgs a{};
-    a.M = T; a.N = V; a.K = H;
-    a.m_tiles = (T + kBM * cta_group() - 1) / (kBM * cta_group());
-    a.n_tiles = (V + kBN - 1) / kBN;
-    a.n_split = pl.n_split;
-    a.tiles_per_split = pl.tiles_per_split;
-    a.kappa = kappa;
-    a.targets = targets;
-    a.partials = partials;
-    a.acc_y = acc_y;
-    a.T_total = T;
-    a.status = status;
-    st = launch_umma<kModeStats>(map_a, map_b, map_a, a, stream);
-    if (st != ULORL_OK) return st;
+    const int tile_m = kBM * cta_group();
+    int chunk = (hooks && hooks->chunk_tokens > 0) ? hooks->chunk_tokens : T;
+    chunk = (chunk + tile_m - 1) / tile_m * tile_m;
+    for (int t0 = 0; t0 < T; t0 += chunk) {
+      const int rows = (T - t0) < chunk ? (T - t0) : chunk;
+      if (hooks && hooks->before_stats_chunk) {
+        st = hooks->before_stats_chunk(t0, rows);
+        if (st != ULORL_OK) return st;
+      }
+      UmmaArgs a{};
+      a.M = rows; a.N = V; a.K = H;
+      a.m_tiles = (rows + tile_m - 1) / tile_m;
+      a.n_tiles = (V + kBN - 1) / kBN;
+      a.n_split = pl.n_split;
+      a.tiles_per_split = pl.tiles_per_split;
+      a.a_mn0 = t0;
+      a.row0 = t0;
+      a.kappa = kappa;
+      a.targets = targets;
+      a.partials = partials;
+      a.acc_y = acc_y;
+      a.T_total = T;
+      a.status = status;
+      st = launch_umma<kModeStats>(map_a, map_b, map_a, a, stream);
+      if (st != ULORL_OK) return st;
+    }
   } else {
+    if (hooks && hooks->before_stats_chunk) {
+      st = hooks->before_stats_chunk(0, T);
+      if (st != ULORL_OK) return st;
+    }
     const dim3 grid((T + kSimtTile - 1) / kSimtTile, pl.n_split);
     if (params->dtype == ULORL_F32)
       simt_stats_kernel<float><<<grid, kSimtThreads, 0, stream>>>(
@@ -453,9 +479,19 @@ int ulorl_token_loss_fwd(const ulorl_params_t* params, const void* hidden, const
                     grad_coef, flags, seq_entropy, loss, stats, ws, stream);
 }
 
-int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const void* W, const int32_t* targets,
-                         const float* lse, const float* grad_coef, const float* grad_loss, void* d_hidden, float* d_W,
+int ulorl_token_loss_fwd(const ulorl_params_t* params, const void* hidden, const void* W, const int32_t* targets,
+                         const float* old_logp, const int32_t* segment_version, const float* advantages,
+                         const int32_t* seq_offsets, const float* entropy_supplied, float* logp, float* entropy,
+                         float* lse, float* grad_coef, uint8_t* flags, float* seq_entropy, float* loss, void* stats,
                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return fwd_impl(params, hidden, W, targets, old_logp, segment_version, advantages, seq_offsets, entropy_supplied, logp,
+                  entropy, lse, grad_coef, flags, seq_entropy, loss, stats, workspace, workspace_bytes, cuda_stream,
+                  nullptr);
+}
+
+static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void* W, const int32_t* targets,
+                    const float* lse, const float* grad_coef, const float* grad_loss, void* d_hidden, float* d_W,
+                    void* workspace, size_t workspace_bytes, void* cuda_stream, const StepHooks* hooks) {
   int st = validate_params(params);
   if (st != ULORL_OK) return st;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
@@ -560,6 +596,10 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
         a.status = status;
         st = launch_umma<kModeDHidden>(map_dz_k, map_w_mn, map_w_mn, a, stream);
         if (st != ULORL_OK) return st;
+        if (hooks && hooks->after_dhidden_panel && !pl.compact) {
+          st = hooks->after_dhidden_panel(t0, rows);
+          if (st != ULORL_OK) return st;
+        }
       }
       // d_W[v, h] (+)= sum_m dz[m, v] hidden[t0 + m, h]
       {
@@ -621,8 +661,19 @@ int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const
           dz, 1, pl.dz_ld, h + (size_t)t0 * H, (size_t)H, 1, d_W, (size_t)H, V, H, rows, acc);
       ULORL_LAUNCH_CHECK();
     }
+    if (hooks && hooks->after_dhidden_panel) {
+      st = hooks->after_dhidden_panel(t0, rows);
+      if (st != ULORL_OK) return st;
+    }
   }
   return ULORL_OK;
+}
+
+int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const void* W, const int32_t* targets,
+                         const float* lse, const float* grad_coef, const float* grad_loss, void* d_hidden, float* d_W,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return bwd_impl(params, hidden, W, targets, lse, grad_coef, grad_loss, d_hidden, d_W, workspace, workspace_bytes,
+                  cuda_stream, nullptr);
 }
 
 // ------------------------------------------------------------------ decision stage without a workspace
@@ -724,6 +775,38 @@ struct HostStepLayout {
   size_t logp, entropy, lse, grad_coef, flags, seq_entropy, loss, stats, d_hidden, d_W, ws, total;
   size_t elem;
 };
+// Two copy streams and a few events, created on the first host-buffer step and kept: the inbound
+// copies run ahead of the forward, the outbound copies of d_hidden behind the backward.
+struct HostStepStreams {
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t start = nullptr, out_done = nullptr;
+  std::vector<cudaEvent_t> chunk_in, panel_out;
+  bool reserve(size_t n) {
+    while (chunk_in.size() < n) {
+      cudaEvent_t e0, e1;
+      if (cudaEventCreateWithFlags(&e0, cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreateWithFlags(&e1, cudaEventDisableTiming) != cudaSuccess)
+        return false;
+      chunk_in.push_back(e0);
+      panel_out.push_back(e1);
+    }
+    return true;
+  }
+};
+HostStepStreams* host_step_streams() {
+  static HostStepStreams hs;
+  static bool ready = false;
+  if (!ready) {
+    if (cudaStreamCreateWithFlags(&hs.in, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&hs.out, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&hs.start, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&hs.out_done, cudaEventDisableTiming) != cudaSuccess)
+      return nullptr;
+    ready = true;
+  }
+  return &hs;
+}
+
 HostStepLayout host_step_layout(const ulorl_params_t* p) {
   HostStepLayout L{};
   const size_t T = (size_t)p->T, H = (size_t)p->H, V = (size_t)p->V, S = (size_t)(p->num_seqs > 0 ? p->num_seqs : 1);
@@ -774,38 +857,78 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   uint8_t* a = reinterpret_cast<uint8_t*>(d_arena);
   const size_t T = (size_t)params->T, H = (size_t)params->H, V = (size_t)params->V, S = (size_t)params->num_seqs;
+  HostStepStreams* hs = host_step_streams();
+  if (!hs) return ULORL_ERR_CUDA;
+  const Plan pl = make_plan(params);
+  const size_t row_bytes = H * L.elem;
+  auto ok = [](cudaError_t e) { return e == cudaSuccess; };
+
+  // copies in, on their own stream, ordered after whatever the caller's stream did to the arena before
+  if (!ok(cudaEventRecord(hs->start, stream)) || !ok(cudaStreamWaitEvent(hs->in, hs->start, 0))) return ULORL_ERR_CUDA;
   auto h2d = [&](size_t off, const void* src, size_t bytes) {
-    return (!src || !bytes) ? cudaSuccess : cudaMemcpyAsync(a + off, src, bytes, cudaMemcpyHostToDevice, stream);
+    return (!src || !bytes) ? cudaSuccess : cudaMemcpyAsync(a + off, src, bytes, cudaMemcpyHostToDevice, hs->in);
   };
+  if (!ok(h2d(L.targets, h_targets, T * 4)) || !ok(h2d(L.old_logp, h_old_logp, T * 4)) ||
+      !ok(h2d(L.segver, h_segment_version, T * 4)) ||
+      !ok(h2d(L.adv, h_advantages, (params->adv_per_token ? T : S) * 4)) ||
+      !ok(h2d(L.seq_off, h_seq_offsets, (S + 1) * 4)) || !ok(h2d(L.ent_sup, h_entropy_supplied, S * 4)) ||
+      !ok(h2d(L.W, h_W, V * H * L.elem)))
+    return ULORL_ERR_CUDA;
+  // hidden states chunk by chunk, one event per chunk: the statistics kernel of a chunk starts as soon as
+  // its rows have landed while the later chunks are still on the bus
+  const int chunk = pl.panel_tokens;
+  const int n_chunks = params->T > 0 ? (params->T + chunk - 1) / chunk : 0;
+  if (!hs->reserve((size_t)n_chunks)) return ULORL_ERR_CUDA;
+  for (int c = 0; c < n_chunks; ++c) {
+    const size_t t0 = (size_t)c * chunk, rows = (T - t0) < (size_t)chunk ? (T - t0) : (size_t)chunk;
+    if (!ok(h2d(L.hidden + t0 * row_bytes, static_cast<const uint8_t*>(h_hidden) + t0 * row_bytes, rows * row_bytes)) ||
+        !ok(cudaEventRecord(hs->chunk_in[c], hs->in)))
+      return ULORL_ERR_CUDA;
+  }
+  StepHooks hooks;
+  hooks.chunk_tokens = chunk;
+  hooks.before_stats_chunk = [&](int t0, int rows) {   // the last chunk that [t0, t0 + rows) touches has landed
+    return ok(cudaStreamWaitEvent(stream, hs->chunk_in[(t0 + rows - 1) / chunk], 0)) ? ULORL_OK : ULORL_ERR_CUDA;
+  };
+  // d_hidden rows of a panel go back on the outbound stream while the next panel is computed
+  hooks.after_dhidden_panel = [&](int t0, int rows) {
+    if (!h_d_hidden) return (int)ULORL_OK;
+    const int c = t0 / chunk;
+    if (!ok(cudaEventRecord(hs->panel_out[c], stream)) || !ok(cudaStreamWaitEvent(hs->out, hs->panel_out[c], 0)) ||
+        !ok(cudaMemcpyAsync(static_cast<uint8_t*>(h_d_hidden) + (size_t)t0 * row_bytes,
+                            a + L.d_hidden + (size_t)t0 * row_bytes, (size_t)rows * row_bytes, cudaMemcpyDeviceToHost,
+                            hs->out)))
+      return (int)ULORL_ERR_CUDA;
+    return (int)ULORL_OK;
+  };
+  st = fwd_impl(params, a + L.hidden, a + L.W, reinterpret_cast<const int32_t*>(a + L.targets),
+                h_old_logp ? reinterpret_cast<const float*>(a + L.old_logp) : nullptr,
+                h_segment_version ? reinterpret_cast<const int32_t*>(a + L.segver) : nullptr,
+                reinterpret_cast<const float*>(a + L.adv), reinterpret_cast<const int32_t*>(a + L.seq_off),
+                h_entropy_supplied ? reinterpret_cast<const float*>(a + L.ent_sup) : nullptr,
+                reinterpret_cast<float*>(a + L.logp), reinterpret_cast<float*>(a + L.entropy),
+                reinterpret_cast<float*>(a + L.lse), reinterpret_cast<float*>(a + L.grad_coef), a + L.flags,
+                reinterpret_cast<float*>(a + L.seq_entropy), reinterpret_cast<float*>(a + L.loss), a + L.stats, a + L.ws,
+                L.total - L.ws, stream, &hooks);
+  if (st != ULORL_OK) return st;
+  // the host buffers are free again once the inbound stream has read them
+  if (!ok(cudaEventRecord(hs->start, hs->in)) || !ok(cudaStreamWaitEvent(stream, hs->start, 0))) return ULORL_ERR_CUDA;
   auto d2h = [&](void* dst, size_t off, size_t bytes) {
     return (!dst || !bytes) ? cudaSuccess : cudaMemcpyAsync(dst, a + off, bytes, cudaMemcpyDeviceToHost, stream);
   };
-  if (h2d(L.hidden, h_hidden, T * H * L.elem) != cudaSuccess || h2d(L.W, h_W, V * H * L.elem) != cudaSuccess ||
-      h2d(L.targets, h_targets, T * 4) != cudaSuccess || h2d(L.old_logp, h_old_logp, T * 4) != cudaSuccess ||
-      h2d(L.segver, h_segment_version, T * 4) != cudaSuccess ||
-      h2d(L.adv, h_advantages, (params->adv_per_token ? T : S) * 4) != cudaSuccess ||
-      h2d(L.seq_off, h_seq_offsets, (S + 1) * 4) != cudaSuccess || h2d(L.ent_sup, h_entropy_supplied, S * 4) != cudaSuccess)
+  if (!ok(d2h(h_logp, L.logp, T * 4)) || !ok(d2h(h_entropy, L.entropy, T * 4)) || !ok(d2h(h_flags, L.flags, T)) ||
+      !ok(d2h(h_seq_entropy, L.seq_entropy, S * 4)) || !ok(d2h(h_loss, L.loss, 4)) ||
+      !ok(d2h(h_stats, L.stats, sizeof(ulorl_stats_t))))
     return ULORL_ERR_CUDA;
-  st = ulorl_token_loss_fwd(params, a + L.hidden, a + L.W, reinterpret_cast<const int32_t*>(a + L.targets),
-                            h_old_logp ? reinterpret_cast<const float*>(a + L.old_logp) : nullptr,
-                            h_segment_version ? reinterpret_cast<const int32_t*>(a + L.segver) : nullptr,
-                            reinterpret_cast<const float*>(a + L.adv), reinterpret_cast<const int32_t*>(a + L.seq_off),
-                            h_entropy_supplied ? reinterpret_cast<const float*>(a + L.ent_sup) : nullptr,
-                            reinterpret_cast<float*>(a + L.logp), reinterpret_cast<float*>(a + L.entropy),
-                            reinterpret_cast<float*>(a + L.lse), reinterpret_cast<float*>(a + L.grad_coef), a + L.flags,
-                            reinterpret_cast<float*>(a + L.seq_entropy), reinterpret_cast<float*>(a + L.loss),
-                            a + L.stats, a + L.ws, L.total - L.ws, stream);
+  st = bwd_impl(params, a + L.hidden, a + L.W, reinterpret_cast<const int32_t*>(a + L.targets),
+                reinterpret_cast<const float*>(a + L.lse), reinterpret_cast<const float*>(a + L.grad_coef), nullptr,
+                a + L.d_hidden, reinterpret_cast<float*>(a + L.d_W), a + L.ws, L.total - L.ws, stream, &hooks);
   if (st != ULORL_OK) return st;
-  st = ulorl_token_loss_bwd(params, a + L.hidden, a + L.W, reinterpret_cast<const int32_t*>(a + L.targets),
-                            reinterpret_cast<const float*>(a + L.lse), reinterpret_cast<const float*>(a + L.grad_coef),
-                            nullptr, a + L.d_hidden, reinterpret_cast<float*>(a + L.d_W), a + L.ws, L.total - L.ws,
-                            stream);
-  if (st != ULORL_OK) return st;
-  if (d2h(h_logp, L.logp, T * 4) != cudaSuccess || d2h(h_entropy, L.entropy, T * 4) != cudaSuccess ||
-      d2h(h_flags, L.flags, T) != cudaSuccess || d2h(h_seq_entropy, L.seq_entropy, S * 4) != cudaSuccess ||
-      d2h(h_loss, L.loss, 4) != cudaSuccess || d2h(h_stats, L.stats, sizeof(ulorl_stats_t)) != cudaSuccess ||
-      d2h(h_d_hidden, L.d_hidden, T * H * L.elem) != cudaSuccess || d2h(h_d_W, L.d_W, V * H * 4) != cudaSuccess)
-    return ULORL_ERR_CUDA;
+  // with compaction d_hidden is only final after the scatter at the end of the backward
+  if (pl.compact && !ok(d2h(h_d_hidden, L.d_hidden, T * row_bytes))) return ULORL_ERR_CUDA;
+  if (!ok(d2h(h_d_W, L.d_W, V * H * 4))) return ULORL_ERR_CUDA;
+  // the caller's stream is done only when the outbound copies are
+  if (!ok(cudaEventRecord(hs->out_done, hs->out)) || !ok(cudaStreamWaitEvent(stream, hs->out_done, 0))) return ULORL_ERR_CUDA;
   return ULORL_OK;
 }
 
