@@ -7,13 +7,18 @@
 //   kModeDHidden d_hidden[t, :] = sum_v dz[t, v] W[v, :]
 //   kModeDW      d_W[v, :] (+)= sum_t dz[t, v] hidden[t, :]
 //
-// One persistent CTA per SM, 192 threads: warp 0 feeds a 4-stage shared-memory ring with TMA tile
-// loads (128-byte swizzle), warp 1 issues tcgen05.mma (128 x 256 x 16 per instruction) into one of
-// two 256-column tensor-memory accumulators, warps 2-5 drain the other accumulator with tcgen05.ld
-// (one token row per thread) and run the mode's epilogue, so the epilogue of tile i overlaps the
-// contraction of tile i + 1.  Operands whose contraction index is not the contiguous one in memory
-// (W and hidden in the two gradient contractions, dz in the d_W one) are loaded as MN-major tiles;
-// nothing is transposed in global memory.
+// One kernel template umma_kernel<mode, CTAs per MMA, accumulators per unit>, persistent, one CTA per
+// SM, 192 threads: one thread of warp 0 feeds a shared-memory ring with TMA tile loads (128-byte
+// swizzle), one thread of warp 1 issues tcgen05.mma into tensor memory, warps 2-5 drain accumulators
+// with tcgen05.ld (one output row per thread) and run the mode's epilogue.
+//   <m, 2, 1>  CTA pair, one 256 x 256 MMA tile over both CTAs, two 256-column accumulator buffers: the
+//              epilogue of tile i overlaps the contraction of tile i + 1 (statistics, dz)
+//   <m, 2, 2>  CTA pair, 256 x 512 unit = two accumulators fed from the same A stage, tensor memory as
+//              one buffer (d_hidden, d_W: long reductions, light epilogues)
+//   <m, 1, 1>  single CTA, 128 x 256 tile, two accumulator buffers (cross-check variant)
+// Operands whose contraction index is not the contiguous one in memory (W and hidden in the two
+// gradient contractions, dz in the d_W one) are loaded as MN-major tiles; nothing is transposed in
+// global memory.  No TMA multicast is used.  Every mbarrier wait is bounded.
 #pragma once
 
 #include "common.cuh"
@@ -38,6 +43,7 @@ constexpr uint32_t kChunkBytes = 64 * kBK * 2;   // one MN-major box: 64 k-rows 
 // for both column blocks (48 KB a stage, 4 stages), eight MMAs are queued per barrier round trip,
 // and tensor memory is used as one 512-column buffer, so the epilogue does not overlap the next
 // unit -- right for the gradient contractions, whose reduction runs over 10^4..10^5 elements.
+
 // Two staging tiles (128 rows x 128 bytes each, 128-byte swizzle) through which the d_W epilogue
 // hands 32-column chunks of the accumulator to TMA store / reduce-add.
 constexpr uint32_t kOutStageBytes = kBM * 128;
