@@ -223,6 +223,11 @@ static int launch_umma_impl(const CUtensorMap& ma, const CUtensorMap& mb, const 
   const int units = (kMode == kModeStats) ? a.m_tiles * a.n_split : a.m_tiles * a.n_tiles;
   if (units <= 0) return ULORL_OK;
   if (kMode != kModeStats && a.group_m <= 0) return ULORL_ERR_INVALID_ARG;
+  // L2 policy of the tile loads: keep what is re-read for long (the hidden tile of the two logits
+  // kernels, the slices of W / of the hidden panel that every pair sweeps in the gradient kernels)
+  UmmaArgs a2 = a;
+  a2.l2_a = (kMode == kModeStats || kMode == kModeDz) ? ptx::kL2EvictLast : ptx::kL2Normal;
+  a2.l2_b = (kMode == kModeDHidden || kMode == kModeDW) ? ptx::kL2EvictLast : ptx::kL2Normal;
   const int max_workers = num_sms / kCta;
   const int workers = units < max_workers ? units : max_workers;
   cudaEvent_t e0 = nullptr, e1 = nullptr;
@@ -243,7 +248,7 @@ static int launch_umma_impl(const CUtensorMap& ma, const CUtensorMap& mb, const 
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  const cudaError_t le = cudaLaunchKernelEx(&cfg, umma_kernel<kMode, kCta, kAcc>, ma, mb, mc, a);
+  const cudaError_t le = cudaLaunchKernelEx(&cfg, umma_kernel<kMode, kCta, kAcc>, ma, mb, mc, a2);
   if (le != cudaSuccess) {
     std::fprintf(stderr, "ulorl: cudaLaunchKernelEx failed: %s\n", cudaGetErrorString(le));
     return ULORL_ERR_CUDA;

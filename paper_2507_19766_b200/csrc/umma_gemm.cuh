@@ -89,6 +89,7 @@ struct UmmaArgs {
   size_t out_ld;
   int accumulate;
   int* status;
+  int l2_a, l2_b;           // ptx::L2Hint of the loads of A and of B (CTA-pair kernels)
   const int* dyn_rows;      // optional device count of rows of the whole (compacted) batch: the launch then
   int dyn_base;             // covers rows [dyn_base, min(dyn_base + capacity, *dyn_rows)) of it (M, or K for d_W)
 };
@@ -271,6 +272,11 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       uint32_t stage = 0, phase = 0;
       uint32_t issued = 0;
       const uint32_t full0 = kPair ? map_to_cta(smem_u32(&bar_full[0]), 0) : smem_u32(&bar_full[0]);
+      // which operand is worth keeping in L2: the hidden tile that a pair re-reads for every vocabulary
+      // tile (statistics, dz), the slices of W / the hidden panel that every pair sweeps (d_hidden, d_W);
+      // the dz stream of the gradient kernels is read by four pairs and then dead
+      const uint64_t pol_a = make_l2_policy(args.l2_a);
+      const uint64_t pol_b = make_l2_policy(args.l2_b);
       for (int unit = worker; unit < n_units; unit += n_workers) {
         int m_tile, n_begin, n_end;
         if (kMode == kModeStats) {
@@ -301,18 +307,18 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
               if (kPair) {
                 if (kAmn) {
 #pragma unroll
-                  for (int j = 0; j < kBM / 64; ++j) tma_load_2d_pair(sa + j * kChunkBytes, &map_a, full, a_row + j * 64, ka);
+                  for (int j = 0; j < kBM / 64; ++j) tma_load_2d_pair(sa + j * kChunkBytes, &map_a, full, a_row + j * 64, ka, pol_a);
                 } else {
-                  tma_load_2d_pair(sa, &map_a, full, ka, a_row);
+                  tma_load_2d_pair(sa, &map_a, full, ka, a_row, pol_a);
                 }
 #pragma unroll
                 for (int q = 0; q < kAcc; ++q) {
                   if (kBmn) {
 #pragma unroll
                     for (int j = 0; j < kBNcta / 64; ++j)
-                      tma_load_2d_pair(sb + q * kBBytesCta + j * kChunkBytes, &map_b, full, b_row + q * kBN + j * 64, kbb);
+                      tma_load_2d_pair(sb + q * kBBytesCta + j * kChunkBytes, &map_b, full, b_row + q * kBN + j * 64, kbb, pol_b);
                   } else {
-                    tma_load_2d_pair(sb + q * kBBytesCta, &map_b, full, kbb, b_row + q * kBN);
+                    tma_load_2d_pair(sb + q * kBBytesCta, &map_b, full, kbb, b_row + q * kBN, pol_b);
                   }
                 }
               } else {
