@@ -86,6 +86,20 @@ static Plan make_plan(const ulorl_params_t* p) {
   want = want < 1 ? 1 : want;
   want = want > kMaxSplits ? kMaxSplits : want;
   want = want > n_tiles ? n_tiles : want;
+  if (pl.tensor && m_tiles > 0) {
+    // persistent kernel: units = row tiles x splits are dealt round-robin to the workers, so the time is
+    // (waves of units) x (vocabulary tiles per split); take the split count from `want` up that wastes least
+    long best_cost = -1;
+    int best = want;
+    for (int s = want; s <= kMaxSplits && s <= n_tiles; ++s) {
+      const int tps = (n_tiles + s - 1) / s;
+      const int s_eff = (n_tiles + tps - 1) / tps;
+      const long waves = ((long)m_tiles * s_eff + workers - 1) / workers;
+      const long cost = waves * tps;
+      if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
+    }
+    want = best;
+  }
   pl.tiles_per_split = (n_tiles + want - 1) / want;
   pl.n_split = (n_tiles + pl.tiles_per_split - 1) / pl.tiles_per_split;
   int panel = p->bwd_panel_tokens > 0 ? p->bwd_panel_tokens
