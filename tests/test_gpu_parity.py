@@ -30,8 +30,12 @@ def gpu_fwd_bwd(batch, gp, grad_loss=None, entropy_supplied=None):
 
 
 def check_against_oracle(batch, gp, op, grad_loss=None, check_grads=True):
+    """Everything the oracle computes comes from the stored inputs only; data flows from the oracle
+    to the GPU (its float32 log-probs into the decision kernel, its coefficients into the backward),
+    never the other way."""
     out, dH, dW = gpu_fwd_bwd(batch, gp, grad_loss=grad_loss)
     oi = oracle_inputs(batch)
+    S = batch.workload.S
     ref = O.forward(oi["hidden"], oi["W"], oi["targets"], oi["old_logp"], oi["segment_version"], oi["advantages"],
                     oi["seq_offsets"], op)
     logp = out.logp.cpu().numpy()
@@ -40,40 +44,59 @@ def check_against_oracle(batch, gp, op, grad_loss=None, check_grads=True):
     assert np.abs(logp - ref["logp"]).max() <= TOL_LOGP
     assert np.abs(ent - ref["entropy"]).max() <= TOL_LOGP
     assert np.abs(lse - ref["lse"]).max() <= TOL_LOGP
-    seq_ent = out.seq_entropy.cpu().numpy()[: batch.workload.S]
+    seq_ent = out.seq_entropy.cpu().numpy()[:S]
     assert np.abs(seq_ent - ref["seq_entropy"]).max() <= TOL_LOGP
+    st = out.stats_host()
+    assert abs(st["mean_entropy"] - ref["mean_entropy"]) <= TOL_LOGP and st["device_status"] == 0
 
-    # decisions: exact wherever the oracle's own value is not within the tolerance of a threshold
+    # (1) fused path: decisions equal the oracle's wherever the oracle's own value is not within the
+    #     tolerance of a threshold; coefficients of the tokens decided alike agree to the log-prob error
     flags = out.flags.cpu().numpy()
     near = near_threshold(ref["logp"], oi["old_logp"], ref["seq_entropy"], oi["seq_offsets"], op)
     differ = flags != ref["flags"]
     assert not (differ & ~near).any(), f"{int((differ & ~near).sum())} decisions differ away from any threshold"
-
-    # decisions and values re-derived by the oracle from the GPU's own float32 log-probs: exact flags
-    gate = O.gate_entropy(ent, oi["seq_offsets"], op.ent_scope)
-    assert np.abs(gate - seq_ent).max() <= 1e-6 or op.ent_scope != "per_seq"
-    dec = O.decide(logp, seq_ent if op.ent_scope == "per_seq" else gate, oi["old_logp"], oi["advantages"],
-                   oi["seq_offsets"], oi["segment_version"], op)
-    assert np.array_equal(flags, dec["flags"])
     g = out.grad_coef.cpu().numpy()
-    assert np.allclose(g, dec["grad_coef"], rtol=2e-6, atol=1e-12)
-    st = out.stats_host()
-    for k in STAT_KEYS:
-        assert st[k] == dec["stats"][k], k
-    assert st["stale_tokens"] == dec["stats"]["stale_tokens"].tolist()
-    assert st["stale_clipped"] == dec["stats"]["stale_clipped"].tolist()
-    assert np.allclose(st["stale_mean_abs_logratio"], dec["stats"]["stale_mean_abs_logratio"], rtol=1e-5, atol=1e-7)
-    assert st["device_status"] == 0
+    same = ~differ
+    assert np.allclose(g[same], ref["grad_coef"][same], rtol=2 * TOL_LOGP, atol=1e-12)
     loss = float(out.loss.cpu()[0])
-    assert abs(loss - dec["loss"]) <= 2e-6 * max(1.0, abs(dec["loss"]))
+    N = float(op.norm_tokens) if op.norm_tokens > 0 else float(batch.workload.T)
+    flip_slack = float(np.abs(ref["surrogate"][differ]).sum()) / N        # what flipped tokens can move
+    assert abs(loss - ref["loss"]) <= TOL_LOSS * max(abs(ref["loss"]), 1e-3) + flip_slack
     if not differ.any():
-        assert abs(loss - ref["loss"]) <= TOL_LOSS * max(abs(ref["loss"]), 1e-3)
-    assert abs(st["mean_entropy"] - ref["mean_entropy"]) <= TOL_LOGP
+        for k in STAT_KEYS:
+            assert st[k] == ref["stats"][k], k
+
+    # (2) decision kernel alone on the oracle's float32 log-probs and entropies: bit-exact flags and counts
+    t = lambda x, dt: torch.from_numpy(np.ascontiguousarray(x)).to(dt).to(DEV)
+    b = batch.to(DEV)
+    dec = B.token_loss_decide(gp, t(ref["logp"].astype(np.float32), torch.float32),
+                              t(ref["entropy"].astype(np.float32), torch.float32), b.old_logp, b.segment_version,
+                              b.advantages, b.seq_offsets)
+    torch.cuda.synchronize()
+    assert np.array_equal(dec.flags.cpu().numpy(), ref["flags"])
+    assert np.allclose(dec.grad_coef.cpu().numpy(), ref["grad_coef"], rtol=2e-6, atol=1e-12)
+    dst = dec.stats_host()
+    for k in STAT_KEYS:
+        assert dst[k] == ref["stats"][k], k
+    assert dst["stale_tokens"] == ref["stats"]["stale_tokens"].tolist()
+    assert dst["stale_clipped"] == ref["stats"]["stale_clipped"].tolist()
+    assert np.allclose(dst["stale_mean_abs_logratio"], ref["stats"]["stale_mean_abs_logratio"], rtol=1e-5, atol=1e-7)
+    assert abs(float(dec.loss.cpu()[0]) - ref["loss"]) <= 2e-6 * max(1.0, abs(ref["loss"]))
+    assert np.allclose(dec.seq_entropy.cpu().numpy()[:S], ref["seq_entropy"], rtol=1e-6, atol=1e-9)
 
     if check_grads:
-        g_ref = dec["grad_coef"] if differ.any() else ref["grad_coef"]
-        dH_ref, dW_ref = O.backward(oi["hidden"], oi["W"], oi["targets"], g_ref, op.inv_temperature,
-                                    grad_loss=1.0 if grad_loss is None else grad_loss)
+        gl = 1.0 if grad_loss is None else grad_loss
+        dH_ref, dW_ref = O.backward(oi["hidden"], oi["W"], oi["targets"], ref["grad_coef"], op.inv_temperature,
+                                    grad_loss=gl)
+        if differ.any():
+            # (3a) some near-threshold token was decided the other way: compare the backward kernels on the
+            #      oracle's coefficients (the GPU's own are covered by (1))
+            ws = B.alloc_workspace(gp, DEV)
+            glt = None if grad_loss is None else torch.tensor([grad_loss], dtype=torch.float32, device=DEV)
+            dH, dW = B.token_loss_bwd(gp, b.hidden, b.W, b.targets, out.lse,
+                                      t(ref["grad_coef"].astype(np.float32), torch.float32), grad_loss=glt,
+                                      workspace=ws)
+            torch.cuda.synchronize()
         eh = rel_l2(dH.float().cpu().numpy(), dH_ref)
         ew = rel_l2(dW.cpu().numpy(), dW_ref)
         assert eh <= TOL_GRAD and ew <= TOL_GRAD, (eh, ew)
@@ -81,7 +104,7 @@ def check_against_oracle(batch, gp, op, grad_loss=None, check_grads=True):
         # stores dz in bf16 (relative error 2^-9 per element, sum_v |dz[t, v]| <= 2 |coef_t|), so
         # |colsum_h| <= 2^-8 sum_t |coef_t| |hidden[t, h]|; the float32 path is held to 1e-5 of that sum
         col = np.abs(dW.double().sum(dim=0).cpu().numpy()).max()
-        coef_sum = float(np.abs(g).sum()) * op.inv_temperature * (1.0 if grad_loss is None else abs(grad_loss))
+        coef_sum = float(np.abs(ref["grad_coef"]).sum()) * op.inv_temperature * abs(gl) * 1.01
         unit = 2.0 ** -8 if (gp.dtype == "bf16" and gp.kernel_path != "simt") else 1e-5
         assert col <= unit * coef_sum * float(np.abs(oi["hidden"]).max()) + 1e-12
     return out, ref
