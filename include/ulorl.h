@@ -165,6 +165,17 @@ int ulorl_token_loss_decide_static(const ulorl_params_t* params,
                                    void* stats, void* cuda_stream);
 
 /*
+ * Group-normalised advantages (Eq. 4) for responses stored group after group (`group_size` responses
+ * per prompt, the last group may be shorter): advantages[i] = (R_i - mean) / std over the group,
+ * population standard deviation, 0 for a group without spread.  keep[i] (optional) is 1 when the
+ * group satisfies the dynamic-sampling constraint of Eq. 7, 0 < #(R == 1) < G.  rewards,
+ * advantages [num_responses] f32 and keep [num_responses] uint8 are device pointers; the result
+ * is what ulorl_token_loss_fwd takes as per-sequence advantages.
+ */
+int ulorl_group_advantages(const float* rewards, int32_t num_responses, int32_t group_size,
+                           float* advantages, uint8_t* keep, void* cuda_stream);
+
+/*
  * Backward (chain rule through Eq. 6): with dz[t,v] = kappa * grad_loss * grad_coef[t] *
  * (1[v = y_t] - exp(z[t,v] - lse[t])), writes d_hidden[T,H] (params->dtype) and d_W[V,H] (f32;
  * added into when params->dw_accumulate).  grad_loss is a device scalar or NULL (= 1).

@@ -11,6 +11,7 @@ by eye:
 
   step 1  logits                z = kappa * hidden @ W^T              (policy of Eq. 6)
   step 2  log-softmax, entropy  logp = z_y - lse ; Hent = -sum p ln p (Eq. 6, Eq. 10 H-bar)
+  (Eq. 4  group-normalised advantages and the dynamic-sampling filter of Eq. 7: group_advantages)
   step 3  mean entropy          H-bar_i = mean over the sequence       (Eq. 10)
   step 4  MPT mask              Eq. 9 and the indicator of Eq. 10
   step 5  importance ratio      SAIS (Eq. 8) or POIS (Section 3.1.2)
@@ -108,6 +109,35 @@ def token_stats(hidden, W, targets, kappa: float = 1.0, rows=None, chunk: int = 
         ent[a:a + chunk] = -(p * lnp).sum(axis=1)
         lse[a:a + chunk] = lse_c
     return logp, ent, lse
+
+
+# --------------------------------------------------------------------------- upstream of step 4: Eq. 4
+def group_advantages(rewards, group_size: int):
+    """Eq. 4: A_i = (R_i - mean(group)) / std(group) over each group of `group_size` consecutive
+    responses to one prompt, and the dynamic-sampling constraint of Eq. 7: a group is kept only if
+    0 < #(reward == 1) < G.  Readings: std is the population standard deviation (the paper does not
+    say which); a group with zero spread gets advantage 0 (it is dropped by the constraint anyway)."""
+    r = _f64(rewards)
+    S = r.shape[0]
+    adv = np.zeros(S)
+    keep = np.zeros(S, dtype=np.uint8)
+    for a in range(0, S, group_size):
+        grp = r[a:a + group_size]
+        G = grp.shape[0]
+        mean = 0.0
+        for x in grp:
+            mean += x
+        mean /= G
+        var = 0.0
+        for x in grp:
+            var += (x - mean) * (x - mean)
+        std = (var / G) ** 0.5
+        n_correct = int(np.count_nonzero(grp == 1.0))
+        kept = 0 < n_correct < G
+        for j in range(G):
+            adv[a + j] = (grp[j] - mean) / std if std > 0 else 0.0
+            keep[a + j] = 1 if kept else 0
+    return adv, keep
 
 
 # --------------------------------------------------------------------------- step 3

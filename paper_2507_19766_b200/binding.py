@@ -62,7 +62,7 @@ class CStats(ctypes.Structure):
 EXPORTS = ("ulorl_workspace_bytes", "ulorl_token_loss_fwd", "ulorl_token_loss_decide", "ulorl_token_loss_bwd",
            "ulorl_check_status", "ulorl_status_string", "ulorl_launch_count", "ulorl_kernel_timing_begin",
            "ulorl_kernel_timing_end", "ulorl_host_step_arena_bytes", "ulorl_token_loss_step_host",
-           "ulorl_token_loss_decide_static")
+           "ulorl_token_loss_decide_static", "ulorl_group_advantages")
 STATIC_MAX_TOKENS, STATIC_MAX_SEQS = 1 << 20, 1 << 16
 KERNEL_KINDS = ("stats", "dz", "d_hidden", "d_W")
 
@@ -87,6 +87,8 @@ def load_library() -> ctypes.CDLL:
     lib.ulorl_token_loss_decide.argtypes = [cp] + [vp] * 12 + [vp, ctypes.c_size_t, vp]
     lib.ulorl_token_loss_decide_static.restype = ctypes.c_int
     lib.ulorl_token_loss_decide_static.argtypes = [cp] + [vp] * 12 + [vp]
+    lib.ulorl_group_advantages.restype = ctypes.c_int
+    lib.ulorl_group_advantages.argtypes = [vp, ctypes.c_int32, ctypes.c_int32, vp, vp, vp]
     lib.ulorl_token_loss_bwd.restype = ctypes.c_int
     lib.ulorl_token_loss_bwd.argtypes = [cp] + [vp] * 8 + [vp, ctypes.c_size_t, vp]
     lib.ulorl_check_status.restype = ctypes.c_int
@@ -337,3 +339,14 @@ def token_loss_step_host(p: Params, arena: torch.Tensor, hidden, W, targets, old
         _hptr(seq_entropy), _hptr(loss), _hptr(stats), _hptr(d_hidden), _hptr(d_W), _ptr(arena), arena.numel(),
         _stream())
     _check(code, "ulorl_token_loss_step_host")
+
+
+def group_advantages(rewards: torch.Tensor, group_size: int):
+    """ulorl_group_advantages: Eq. 4 advantages and the Eq. 7 keep flag per response (device tensors)."""
+    _want(rewards, torch.float32, rewards.numel(), "rewards")
+    adv = torch.empty_like(rewards)
+    keep = torch.empty(rewards.numel(), dtype=torch.uint8, device=rewards.device)
+    code = load_library().ulorl_group_advantages(_ptr(rewards), rewards.numel(), group_size, _ptr(adv), _ptr(keep),
+                                                 _stream())
+    _check(code, "ulorl_group_advantages")
+    return adv, keep

@@ -256,6 +256,38 @@ __global__ void finalize_kernel(int T, int n_blocks, double inv_N, const DecideP
 }
 
 // ------------------------------------------------------------------------------------------
+// Group-normalised advantages (Eq. 4) and the dynamic-sampling filter of Eq. 7, one thread per
+// group of `group` consecutive responses: A_i = (R_i - mean) / std with the population standard
+// deviation in float64, 0 when the group has no spread; keep_i = 0 < #(R == 1) < G.
+// ------------------------------------------------------------------------------------------
+__global__ void group_advantage_kernel(int S, int group, const float* __restrict__ rewards, float* __restrict__ adv,
+                                       uint8_t* __restrict__ keep) {
+  const int gidx = blockIdx.x * blockDim.x + threadIdx.x;
+  const int a = gidx * group;
+  if (a >= S) return;
+  const int b = min(S, a + group);
+  const int G = b - a;
+  double mean = 0.0;
+  int n_correct = 0;
+  for (int i = a; i < b; ++i) {
+    mean += (double)rewards[i];
+    n_correct += rewards[i] == 1.f ? 1 : 0;
+  }
+  mean /= (double)G;
+  double var = 0.0;
+  for (int i = a; i < b; ++i) {
+    const double d = (double)rewards[i] - mean;
+    var += d * d;
+  }
+  const double sd = sqrt(var / (double)G);
+  const uint8_t kept = (n_correct > 0 && n_correct < G) ? 1 : 0;
+  for (int i = a; i < b; ++i) {
+    adv[i] = sd > 0.0 ? (float)(((double)rewards[i] - mean) / sd) : 0.f;
+    if (keep) keep[i] = kept;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // Active-row compaction of the backward.  Tokens whose d loss / d logp is exactly zero (masked
 // well-mastered positive tokens of Eq. 10, clipped tokens, zero advantage) add nothing to dHidden or
 // dW, so the backward contractions run on the remaining rows only.

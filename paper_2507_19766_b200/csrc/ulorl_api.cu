@@ -762,6 +762,17 @@ int ulorl_token_loss_decide_static(const ulorl_params_t* params, const float* lo
                     grad_coef, flags, seq_entropy, loss, stats, ws, stream);
 }
 
+int ulorl_group_advantages(const float* rewards, int32_t num_responses, int32_t group_size, float* advantages,
+                           uint8_t* keep, void* cuda_stream) {
+  if (num_responses < 0 || group_size <= 0) return ULORL_ERR_INVALID_ARG;
+  if (num_responses == 0) return ULORL_OK;
+  if (!rewards || !advantages) return ULORL_ERR_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const int groups = (num_responses + group_size - 1) / group_size;
+  group_advantage_kernel<<<(groups + 127) / 128, 128, 0, stream>>>(num_responses, group_size, rewards, advantages, keep);
+  return check_launch();
+}
+
 int ulorl_kernel_timing_begin(void) {
   for (int k = 0; k < 4; ++k) g_timing.used[k] = 0;
   g_timing.enabled = true;

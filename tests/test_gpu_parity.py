@@ -457,3 +457,13 @@ def test_inconsistent_sequence_offsets_are_reported_not_followed():
     out = B.token_loss_fwd(gp, b.hidden, b.W, b.targets, b.old_logp, b.segment_version, b.advantages, b.seq_offsets,
                            workspace=ws)
     assert B.check_status(ws) == B.OK
+
+
+def test_group_advantages_match_the_oracle():
+    rng = np.random.default_rng(3)
+    for S, G, p in ((1024, 8, 0.3), (37, 16, 0.5), (5, 8, 0.9), (64, 4, 0.0)):
+        r = (rng.random(S) < p).astype(np.float32)
+        adv, keep = B.group_advantages(torch.from_numpy(r).to(DEV), G)
+        ref_adv, ref_keep = O.group_advantages(r, G)
+        assert np.array_equal(keep.cpu().numpy(), ref_keep)
+        assert np.allclose(adv.cpu().numpy(), ref_adv, rtol=1e-6, atol=1e-7)

@@ -483,3 +483,21 @@ def test_backward_row_subset_and_grad_loss():
     _, dW_a = O.backward(hidden, W, targets, g, rows=np.arange(0, 17))
     _, dW_b = O.backward(hidden, W, targets, g, rows=np.arange(17, 40))
     assert np.allclose(dW_a + dW_b, dW, atol=1e-13)
+
+
+# ------------------------------------------------------------------ Eq. 4 advantages
+def test_group_advantages_closed_forms():
+    # k correct of G with 0/1 rewards: mean p = k/G, std sqrt(p(1-p)); A(1) = sqrt((1-p)/p), A(0) = -sqrt(p/(1-p))
+    r = np.array([1, 0, 0, 0, 1, 1, 1, 1, 0, 0, 0, 0], dtype=np.float32)
+    adv, keep = O.group_advantages(r, 4)
+    assert np.allclose(adv[:4], [math.sqrt(3.0), -math.sqrt(1 / 3), -math.sqrt(1 / 3), -math.sqrt(1 / 3)], atol=1e-15)
+    assert np.array_equal(adv[4:], np.zeros(8))                  # all right / all wrong: no spread
+    assert keep.tolist() == [1] * 4 + [0] * 8                     # Eq. 7: 0 < #correct < G
+    # sign of the advantage is the correctness (Section 3.3); zero mean and unit spread within a kept group
+    r = np.array([1, 1, 0, 1, 0, 0, 1, 0], dtype=np.float32)
+    adv, keep = O.group_advantages(r, 8)
+    assert ((adv > 0) == (r == 1)).all() and abs(adv.mean()) < 1e-15 and abs(adv.std() - 1.0) < 1e-15
+    assert keep.all()
+    # library second opinion
+    ref = (r - r.mean()) / r.std()
+    assert np.allclose(adv, ref, atol=1e-15)
