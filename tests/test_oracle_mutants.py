@@ -29,6 +29,9 @@ MUTANTS = {
     "clipped tokens keep their gradient": ("g = -(1.0 / N) * keep * A * r * (0.0 if (hi or lo) else 1.0)", "g = -(1.0 / N) * keep * A * r"),
     "ratio inverted": ("d32 = np.float32(logp32[t] - np.float32(old_logp[t]))", "d32 = np.float32(np.float32(old_logp[t]) - logp32[t])"),
     "masked tokens keep their gradient": ("g = -(1.0 / N) * keep * A * r *", "g = -(1.0 / N) * A * r *"),
+    "sample std in the advantages": ("std = (var / G) ** 0.5", "std = (var / (G - 1)) ** 0.5"),
+    "advantage sign": ("adv[a + j] = (grp[j] - mean) / std if std > 0 else 0.0", "adv[a + j] = (mean - grp[j]) / std if std > 0 else 0.0"),
+    "group filter keeps all-correct groups": ("kept = 0 < n_correct < G", "kept = 0 < n_correct <= G"),
     "sequence mean divides by T": ("seq_mean[i] = tot / (b - a)", "seq_mean[i] = tot / e.shape[0]"),
 }
 
@@ -46,6 +49,7 @@ PIN_TESTS = [
     lambda: pins.test_dW_column_sums_vanish_and_dhidden_row_form(),
     lambda: [pins.test_finite_differences(k) for k in (1.0, 1.0 / 0.85)],
     lambda: pins.test_staleness_statistics(),
+    lambda: pins.test_group_advantages_closed_forms(),
 ]
 
 
