@@ -104,3 +104,39 @@ def pack_experience(samples: Sequence[Sample], advantages: Sequence[float]):
     current_version = int(version.max()) if version.size else 0
     return dict(targets=targets, old_logp=old_logp, segment_version=version, seq_offsets=seq_offsets,
                 advantages=adv, current_version=current_version)
+
+
+def balance_into_calls(lengths: Sequence[int], max_tokens_per_call: int) -> List[List[int]]:
+    """Split finished samples into calls of at most `max_tokens_per_call` tokens each, whole samples only,
+    with near-equal token counts: the long-tailed length mix of ultra-long rollouts otherwise leaves one
+    call (or one data-parallel rank) holding the few longest samples.  The number of calls is the least
+    that the capacity allows for a first-fit-decreasing packing; samples are then dealt longest first to
+    the lightest call that still has room.  Returns the sample indices of each call, each list ascending.
+    A sample longer than the capacity is an error."""
+    order = sorted(range(len(lengths)), key=lambda i: (-int(lengths[i]), i))
+    if any(int(lengths[i]) > max_tokens_per_call for i in order):
+        raise ValueError("a sample is longer than max_tokens_per_call")
+    bins: List[int] = []                                   # first-fit decreasing fixes the number of calls
+    for i in order:
+        for b in range(len(bins)):
+            if bins[b] + int(lengths[i]) <= max_tokens_per_call:
+                bins[b] += int(lengths[i])
+                break
+        else:
+            bins.append(int(lengths[i]))
+    n_calls = len(bins)
+    while True:
+        load = [0] * n_calls
+        calls: List[List[int]] = [[] for _ in range(n_calls)]
+        ok = True
+        for i in order:
+            fits = [b for b in range(n_calls) if load[b] + int(lengths[i]) <= max_tokens_per_call]
+            if not fits:
+                ok = False
+                break
+            b = min(fits, key=lambda c: (load[c], c))
+            load[b] += int(lengths[i])
+            calls[b].append(i)
+        if ok:
+            return [sorted(c) for c in calls]
+        n_calls += 1                                       # balancing can need one call more than first-fit

@@ -166,6 +166,10 @@ def _sequence_lengths(wl: Workload, rng: np.random.Generator) -> np.ndarray:
         alpha, cap = float(kind[1]), int(kind[2])
         raw = (1.0 - rng.random(wl.S)) ** (-1.0 / alpha)
         return _rescale_to_sum(raw, wl.T, min(cap, wl.T))
+    if kind[0] == "fixed":                       # "fixed:50,25,15": the lengths as given (tests)
+        x = np.array([int(v) for v in kind[1].split(",")], dtype=np.int64)
+        assert x.shape[0] == wl.S and int(x.sum()) == wl.T
+        return x
     raise ValueError(wl.lengths)
 
 

@@ -467,3 +467,60 @@ def test_group_advantages_match_the_oracle():
         ref_adv, ref_keep = O.group_advantages(r, G)
         assert np.array_equal(keep.cpu().numpy(), ref_keep)
         assert np.allclose(adv.cpu().numpy(), ref_adv, rtol=1e-6, atol=1e-7)
+
+
+def test_token_range_split_with_entropy_exchange_matches_the_unsplit_batch():
+    """Two token ranges of one batch, run one after the other as two ranks would run them: forward on each
+    range, per-sequence (entropy sum, count) partials summed, decision stage with the means supplied,
+    backward accumulating into one d_W.  Flags, loss and gradients equal the unsplit run's."""
+    import dataclasses
+    from paper_2507_19766_b200 import dp
+    wl = synth.WORKLOADS["small"].scaled(T=1500, S=4, H=128, V=1500, lengths="fixed:700,400,300,100", planted=0.6,
+                                         beta_planted=(200.0, 450.0), mpt_mode="dynamic", adv="bern:0.5:3")
+    batch = synth.make_batch(wl, seed=26)
+    gp, op = both_params(batch)
+    oi = oracle_inputs(batch)
+    ref = O.forward(oi["hidden"], oi["W"], oi["targets"], oi["old_logp"], oi["segment_version"], oi["advantages"],
+                    oi["seq_offsets"], op)
+    hbar = np.sort(ref["seq_entropy"])
+    sigma = float(0.5 * (hbar[1] + hbar[2]))                    # gate open for two sequences, shut for two
+    assert min(hbar[2] - sigma, sigma - hbar[1]) > 10 * TOL_LOGP
+    gp, op = both_params(batch, entropy_target=sigma)
+    full, dH_full, dW_full = gpu_fwd_bwd(batch, gp)
+    b = batch.to(DEV)
+    off = batch.seq_offsets.numpy()
+    ranges = dp.shard_token_ranges(wl.T, 2, align=256)
+    assert ranges == [(0, 768), (768, 1500)]                   # sequences 0 and 1 are both split
+    pieces, partial = [], torch.zeros(wl.S, 2, dtype=torch.float64, device=DEV)
+    for lo, hi in ranges:
+        ids, loff = dp.local_sequence_pieces(off, lo, hi)
+        lp = dataclasses.replace(gp, T=hi - lo, num_seqs=len(ids), norm_tokens=wl.T, ent_scope="supplied",
+                                 dw_accumulate=True)
+        loff_t = torch.tensor(loff, dtype=torch.int32, device=DEV)
+        adv = b.advantages[torch.tensor(ids, device=DEV)].contiguous()
+        dummy = torch.zeros(len(ids), dtype=torch.float32, device=DEV)
+        sl = slice(lo, hi)
+        f = B.token_loss_fwd(lp, b.hidden[sl], b.W, b.targets[sl], b.old_logp[sl], b.segment_version[sl], adv, loff_t,
+                             entropy_supplied=dummy)
+        cnt = torch.tensor(np.diff(loff), device=DEV)
+        partial += dp.sequence_entropy_partials(f.seq_entropy[:len(ids)], cnt, ids, wl.S)
+        pieces.append((sl, ids, lp, loff_t, adv, f))
+    dW = torch.zeros(wl.V, wl.H, dtype=torch.float32, device=DEV)
+    dH = torch.empty_like(b.hidden)
+    loss, flags = 0.0, np.zeros(wl.T, dtype=np.uint8)
+    for sl, ids, lp, loff_t, adv, f in pieces:
+        gate = dp.sequence_entropy_from_partials(partial, ids)
+        d = B.token_loss_decide(lp, f.logp, f.entropy, b.old_logp[sl], b.segment_version[sl], adv, loff_t,
+                                entropy_supplied=gate)
+        B.token_loss_bwd(lp, b.hidden[sl], b.W, b.targets[sl], f.lse, d.grad_coef, d_hidden=dH[sl], d_W=dW)
+        loss += float(d.loss.cpu()[0])
+        flags[sl] = d.flags.cpu().numpy()
+    torch.cuda.synchronize()
+    gate_all = dp.sequence_entropy_from_partials(partial, range(wl.S)).cpu().numpy()
+    assert np.abs(gate_all - ref["seq_entropy"]).max() <= TOL_LOGP
+    assert np.array_equal(flags, full.flags.cpu().numpy())
+    masked = (flags & O.FLAG_MASKED) != 0
+    assert 0 < masked.sum() < ((flags & O.FLAG_MPT) != 0).sum()
+    assert abs(loss - float(full.loss.cpu()[0])) <= 1e-5 * max(1e-3, abs(loss))
+    assert torch.equal(dH, dH_full)                            # rows are independent of the split
+    assert rel_l2(dW.cpu().numpy(), dW_full.cpu().numpy()) <= 1e-4

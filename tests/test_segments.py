@@ -81,3 +81,24 @@ def test_rejects_bad_engine_and_bad_config():
         r.step(lambda s, m, v: [([1] * 5, [0.0] * 5, False)], [0], 1, 0)      # 5 tokens in a 4-token segment
     with pytest.raises(ValueError):
         r.step(lambda s, m, v: [], [0], 1, 0)
+
+
+def test_balance_into_calls():
+    from paper_2507_19766_b200.segments import balance_into_calls
+    lengths = [100, 10, 10, 10, 60, 40, 30, 20, 20]            # 300 tokens
+    calls = balance_into_calls(lengths, 150)
+    assert sorted(i for c in calls for i in c) == list(range(9))            # a partition
+    loads = [sum(lengths[i] for i in c) for c in calls]
+    assert len(calls) == 2 and loads == [150, 150]
+    assert all(c == sorted(c) for c in calls)
+    # long tail: capacity forces three calls; each within capacity, spread no worse than the largest sample
+    rng = np.random.default_rng(5)
+    lengths = np.minimum(131072, (2048 * rng.pareto(1.2, size=200) + 256).astype(np.int64)).tolist()
+    calls = balance_into_calls(lengths, 131072)
+    loads = [sum(lengths[i] for i in c) for c in calls]
+    assert sorted(i for c in calls for i in c) == list(range(200))
+    assert max(loads) <= 131072 and len(calls) >= -(-sum(lengths) // 131072)
+    assert max(loads) - min(loads) <= max(lengths)
+    assert balance_into_calls([], 10) == []
+    with pytest.raises(ValueError):
+        balance_into_calls([11], 10)
