@@ -68,6 +68,8 @@ class OracleParams:
     entropy_target: float = 0.2      # sigma, Section 4.1
     inv_temperature: float = 1.0     # kappa
     norm_tokens: int = 0             # N of Eq. 10; 0 means the T tokens of the call
+    loss_norm: str = "tokens"        # "tokens": 1 / sum_i |o_i| (Eq. 7, Eq. 10) | "sequence": (1/G) sum_i 1/|o_i| (Eq. 5)
+    norm_seqs: int = 0               # G of Eq. 5 in "sequence" mode; 0 means the sequences of the call
     current_version: int = 0
 
 
@@ -206,7 +208,10 @@ def decide(logp32, gate_ent32, old_logp, advantages, seq_offsets, segment_versio
     adv_in = np.asarray(advantages, dtype=np.float32)
     ln_tau, ln_hi, ln_lo = decision_thresholds(p)
     sigma32 = np.float32(p.entropy_target)
-    N = float(p.norm_tokens) if p.norm_tokens > 0 else float(T)
+    if p.loss_norm == "tokens":      # one weight 1/N for every token (Eq. 10)
+        N = float(p.norm_tokens) if p.norm_tokens > 0 else float(T)
+    else:                            # GRPO's per-sample mean (Eq. 5): token of sequence i weighs 1 / (G |o_i|)
+        N = float(p.norm_seqs) if p.norm_seqs > 0 else float(S)
     eps_hi = float(np.float32(p.clip_eps_high))
     eps_lo = float(np.float32(p.clip_eps_low))
 
@@ -223,6 +228,7 @@ def decide(logp32, gate_ent32, old_logp, advantages, seq_offsets, segment_versio
             gate = bool(gate_ent32[i] < sigma32)          # strict, as printed in Eq. 10
         else:
             gate = False
+        wlen = 1.0 if p.loss_norm == "tokens" else 1.0 / max(1.0, float(off[i + 1] - off[i]))
         for t in range(int(off[i]), int(off[i + 1])):
             A32 = adv_in[t] if adv_per_token else adv_in[i]
             A = float(A32)
@@ -242,9 +248,9 @@ def decide(logp32, gate_ent32, old_logp, advantages, seq_offsets, segment_versio
             c = min(max(r, 1.0 - eps_lo), 1.0 + eps_hi)
             s = min(r * A, c * A)
             keep = 0.0 if msk else 1.0
-            loss_sum += keep * s
+            loss_sum += keep * s * wlen
             # step 7
-            g = -(1.0 / N) * keep * A * r * (0.0 if (hi or lo) else 1.0)
+            g = -(1.0 / N) * keep * A * r * (0.0 if (hi or lo) else 1.0) * wlen
             f = 0
             if msk:
                 f |= FLAG_MASKED
@@ -361,14 +367,22 @@ def objective_value(hidden, W, targets, old_logp, advantages, seq_offsets, maske
     off = np.asarray(seq_offsets, dtype=np.int64)
     adv_in = np.asarray(advantages, dtype=np.float64)
     N = float(p.norm_tokens) if p.norm_tokens > 0 else float(T)
+    G = float(p.norm_seqs) if p.norm_seqs > 0 else float(off.shape[0] - 1)
     eps_hi = float(np.float32(p.clip_eps_high))
     eps_lo = float(np.float32(p.clip_eps_low))
     tot = 0.0
+    per_sample = 0.0
     for i in range(off.shape[0] - 1):
+        seq = 0.0
         for t in range(int(off[i]), int(off[i + 1])):
             A = float(adv_in[t] if adv_per_token else adv_in[i])
             r = float(np.exp(logp[t] - float(old_logp[t])))
             c = min(max(r, 1.0 - eps_lo), 1.0 + eps_hi)
             if not masked[t]:
-                tot += min(r * A, c * A)
+                seq += min(r * A, c * A)
+        tot += seq
+        if off[i + 1] > off[i]:
+            per_sample += seq / float(off[i + 1] - off[i])
+    if p.loss_norm == "sequence":    # Eq. 5: mean over the group of each sample's token mean
+        return -per_sample / G
     return -tot / N

@@ -32,6 +32,9 @@ MUTANTS = {
     "sample std in the advantages": ("std = (var / G) ** 0.5", "std = (var / (G - 1)) ** 0.5"),
     "advantage sign": ("adv[a + j] = (grp[j] - mean) / std if std > 0 else 0.0", "adv[a + j] = (mean - grp[j]) / std if std > 0 else 0.0"),
     "group filter keeps all-correct groups": ("kept = 0 < n_correct < G", "kept = 0 < n_correct <= G"),
+    "per-sample weight forgotten in the gradient": ("(0.0 if (hi or lo) else 1.0) * wlen", "(0.0 if (hi or lo) else 1.0)"),
+    "per-sample weight uses T": ("1.0 / max(1.0, float(off[i + 1] - off[i]))", "1.0 / float(T)"),
+    "per-sample mode divides by tokens": ("N = float(p.norm_seqs) if p.norm_seqs > 0 else float(S)\n    eps_hi", "N = float(T)\n    eps_hi"),
     "sequence mean divides by T": ("seq_mean[i] = tot / (b - a)", "seq_mean[i] = tot / e.shape[0]"),
 }
 
@@ -47,9 +50,11 @@ PIN_TESTS = [
     lambda: pins.test_entropy_scopes_and_sequence_means(),
     lambda: pins.test_mean_nll_special_case(),
     lambda: pins.test_dW_column_sums_vanish_and_dhidden_row_form(),
-    lambda: [pins.test_finite_differences(k) for k in (1.0, 1.0 / 0.85)],
+    lambda: [pins.test_finite_differences(k, "tokens") for k in (1.0, 1.0 / 0.85)],
     lambda: pins.test_staleness_statistics(),
     lambda: pins.test_group_advantages_closed_forms(),
+    lambda: pins.test_sequence_normalisation_closed_forms(),
+    lambda: pins.test_finite_differences(1.0, "sequence"),
 ]
 
 

@@ -416,8 +416,8 @@ def test_dW_column_sums_vanish_and_dhidden_row_form():
     assert np.allclose(out["d_hidden"], expect, atol=1e-12)
 
 
-@pytest.mark.parametrize("kappa", [1.0, 1.0 / 0.85])
-def test_finite_differences(kappa):
+@pytest.mark.parametrize("kappa,loss_norm", [(1.0, "tokens"), (1.0 / 0.85, "tokens"), (1.0, "sequence")])
+def test_finite_differences(kappa, loss_norm):
     """Central differences of the Eq. 10 objective in float64 on a tiny problem, with clipped,
     masked, negative-advantage and zero-advantage tokens present and every token at least
     1e-2 away from each threshold."""
@@ -436,7 +436,8 @@ def test_finite_differences(kappa):
     logp, _, _ = O.token_stats(hidden, W, targets, kappa)
     shift = np.array([0.0, 0.4, -0.1, -0.5, 0.15, 0.0])     # clip-high on 1, clip-low on 3
     old = (logp - shift).astype(np.float32)
-    p = O.OracleParams(is_mode="sais", mpt_mode="always", inv_temperature=kappa, norm_tokens=9)
+    p = O.OracleParams(is_mode="sais", mpt_mode="always", inv_temperature=kappa, norm_tokens=9, loss_norm=loss_norm,
+                       norm_seqs=4)
     out = O.fwd_bwd(hidden, W, targets, old, np.zeros(T, np.int32), adv, offsets, p)
     fl = out["flags"]
     assert fl[0] & O.FLAG_MASKED and fl[1] & O.FLAG_CLIP_HIGH and fl[3] & O.FLAG_CLIP_LOW
@@ -483,6 +484,34 @@ def test_backward_row_subset_and_grad_loss():
     _, dW_a = O.backward(hidden, W, targets, g, rows=np.arange(0, 17))
     _, dW_b = O.backward(hidden, W, targets, g, rows=np.arange(17, 40))
     assert np.allclose(dW_a + dW_b, dW, atol=1e-13)
+
+
+# ------------------------------------------------------------------ Eq. 5 per-sample normalisation
+def test_sequence_normalisation_closed_forms():
+    """With the ratio identically one and no mask the surrogate of a token is its advantage, so the two
+    normalisations have closed forms: tokens -sum_i |o_i| A_i / T (Eq. 10's 1/sum|o_i|), sequence -(1/G) sum_i A_i
+    (Eq. 5's (1/G) sum_i (1/|o_i|) sum_t), the second independent of the lengths."""
+    off = np.array([0, 7, 9, 12], np.int32)
+    adv = np.array([0.5, -2.0, 1.25], np.float32)
+    T = 12
+    lp = np.full(T, -1.0, np.float32)
+    ent = np.ones(T, np.float32)
+    kw = dict(is_mode="pois", mpt_mode="off")
+    tok = O.decide(lp, ent[:3], None, adv, off, None, O.OracleParams(**kw))
+    seq = O.decide(lp, ent[:3], None, adv, off, None, O.OracleParams(loss_norm="sequence", **kw))
+    assert abs(tok["loss"] + (7 * 0.5 - 2 * 2.0 + 3 * 1.25) / 12) < 1e-15
+    assert abs(seq["loss"] + (0.5 - 2.0 + 1.25) / 3) < 1e-15
+    assert np.allclose(tok["grad_coef"], -np.repeat(adv, [7, 2, 3]) / 12, atol=1e-16)
+    assert np.allclose(seq["grad_coef"], -np.repeat(adv / np.array([7, 2, 3]), [7, 2, 3]) / 3, atol=1e-16)
+    assert np.array_equal(tok["flags"], seq["flags"])                   # decisions do not depend on the weights
+    # G supplied by the caller (a micro-batch of a larger group)
+    seq6 = O.decide(lp, ent[:3], None, adv, off, None, O.OracleParams(loss_norm="sequence", norm_seqs=6, **kw))
+    assert abs(seq6["loss"] - seq["loss"] / 2) < 1e-15 and np.allclose(seq6["grad_coef"], seq["grad_coef"] / 2)
+    # equal lengths: the two normalisations coincide
+    off2 = np.array([0, 4, 8, 12], np.int32)
+    a = O.decide(lp, ent[:3], None, adv, off2, None, O.OracleParams(**kw))
+    b = O.decide(lp, ent[:3], None, adv, off2, None, O.OracleParams(loss_norm="sequence", **kw))
+    assert abs(a["loss"] - b["loss"]) < 1e-15 and np.allclose(a["grad_coef"], b["grad_coef"], atol=1e-16)
 
 
 # ------------------------------------------------------------------ Eq. 4 advantages
