@@ -57,6 +57,11 @@ typedef enum { ULORL_PATH_AUTO = 0, ULORL_PATH_SIMT = 1, ULORL_PATH_TENSOR = 2 }
 
 #define ULORL_N_STALENESS 16
 
+/* Normalisation of the loss.  TOKENS: every response token weighs 1/N, N = all response tokens
+ * (Eq. 7 and Eq. 10, the paper's method).  SEQUENCE: a token of sequence i weighs 1/(G |o_i|), the
+ * per-sample mean of Eq. 5 (GRPO); |o_i| is taken from seq_offsets, so sequences must be whole. */
+typedef enum { ULORL_NORM_TOKENS = 0, ULORL_NORM_SEQUENCE = 1 } ulorl_loss_norm_t;
+
 typedef struct {
   int32_t T, H, V, num_seqs;   /* packed tokens, hidden size, vocabulary, sequences (seq_offsets[num_seqs] == T) */
   int32_t dtype;               /* ulorl_dtype_t of hidden, W, d_hidden                                           */
@@ -79,6 +84,8 @@ typedef struct {
                                /* to either gradient, Eq. 10); results are the same, the workspace grows by two  */
                                /* [T, H] copies.  0 = all rows.  Part of the workspace size: pass the same value */
                                /* to ulorl_workspace_bytes and to both calls.                                    */
+  int32_t loss_norm;           /* ulorl_loss_norm_t: weight of a token's term in the loss                        */
+  int32_t norm_seqs;           /* G of Eq. 5 for ULORL_NORM_SEQUENCE; 0 means num_seqs                           */
 } ulorl_params_t;
 
 typedef struct {

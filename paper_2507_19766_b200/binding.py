@@ -28,6 +28,7 @@ N_STALENESS = 16
 _IS = {"sais": IS_SAIS, "pois": IS_POIS}
 _MPT = {"off": MPT_OFF, "always": MPT_ALWAYS, "dynamic": MPT_DYNAMIC}
 _ENT = {"per_seq": ENT_PER_SEQ, "batch": ENT_BATCH, "supplied": ENT_SUPPLIED}
+_NORM = {"tokens": 0, "sequence": 1}
 _PATH = {"auto": PATH_AUTO, "simt": PATH_SIMT, "tensor": PATH_TENSOR}
 
 
@@ -44,7 +45,7 @@ class CParams(ctypes.Structure):
         ("entropy_target", ctypes.c_float), ("inv_temperature", ctypes.c_float),
         ("norm_tokens", ctypes.c_int64), ("current_version", ctypes.c_int32),
         ("dw_accumulate", ctypes.c_int32), ("kernel_path", ctypes.c_int32), ("bwd_panel_tokens", ctypes.c_int32),
-        ("compact_rows", ctypes.c_int32),
+        ("compact_rows", ctypes.c_int32), ("loss_norm", ctypes.c_int32), ("norm_seqs", ctypes.c_int32),
     ]
 
 
@@ -141,13 +142,16 @@ class Params:
     kernel_path: str = "auto"
     bwd_panel_tokens: int = 0
     compact_rows: bool = False
+    loss_norm: str = "tokens"
+    norm_seqs: int = 0
 
     def to_c(self) -> CParams:
         return CParams(self.T, self.H, self.V, self.num_seqs, BF16 if self.dtype == "bf16" else F32,
                        _IS[self.is_mode], _MPT[self.mpt_mode], _ENT[self.ent_scope], int(self.adv_per_token),
                        self.clip_eps_low, self.clip_eps_high, self.mpt_tau, self.entropy_target,
                        self.inv_temperature, self.norm_tokens, self.current_version, int(self.dw_accumulate),
-                       _PATH[self.kernel_path], self.bwd_panel_tokens, int(self.compact_rows))
+                       _PATH[self.kernel_path], self.bwd_panel_tokens, int(self.compact_rows),
+                       _NORM[self.loss_norm], self.norm_seqs)
 
 
 def workspace_bytes(p: Params) -> int:

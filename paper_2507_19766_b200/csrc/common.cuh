@@ -32,7 +32,7 @@ struct DecidePartial {
 struct DecideConsts {
   float ln_tau, ln_hi, ln_lo, sigma;
   double eps_lo, eps_hi, inv_N;
-  int is_mode, mpt_mode, ent_scope, adv_per_token, current_version;
+  int is_mode, mpt_mode, ent_scope, adv_per_token, current_version, loss_norm;
 };
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

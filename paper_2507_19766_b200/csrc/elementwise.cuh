@@ -140,8 +140,15 @@ __global__ void decide_kernel(int T, int S, DecideConsts c, const float* __restr
     const double Ad = (double)A;
     const double cl = fmin(fmax(r, 1.0 - c.eps_lo), 1.0 + c.eps_hi);
     const double s = fmin(r * Ad, cl * Ad);
-    if (!msk) contrib = s;
-    const double g = (msk || hi || lo) ? 0.0 : -c.inv_N * Ad * r;
+    // weight of the token's term: 1/N (Eq. 10), or 1/(G |o_i|) for the per-sample mean of Eq. 5
+    // (inv_N then holds 1/G)
+    double wlen = 1.0;
+    if (c.loss_norm == ULORL_NORM_SEQUENCE) {
+      const int len = seq_offsets[i + 1] - seq_offsets[i];
+      wlen = 1.0 / (double)(len > 0 ? len : 1);
+    }
+    if (!msk) contrib = s * wlen;
+    const double g = (msk || hi || lo) ? 0.0 : -c.inv_N * Ad * r * wlen;
     const float g32 = (float)g;
     if (grad_coef) grad_coef[t] = g32;
     const unsigned f = (msk ? ULORL_FLAG_MASKED : 0u) | (hi ? ULORL_FLAG_CLIP_HIGH : 0u) |

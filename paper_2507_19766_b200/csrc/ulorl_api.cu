@@ -62,6 +62,8 @@ static int validate_params(const ulorl_params_t* p) {
   if (p->is_mode != ULORL_IS_SAIS && p->is_mode != ULORL_IS_POIS) return ULORL_ERR_INVALID_ARG;
   if (p->mpt_mode < ULORL_MPT_OFF || p->mpt_mode > ULORL_MPT_DYNAMIC) return ULORL_ERR_INVALID_ARG;
   if (p->ent_scope < ULORL_ENT_PER_SEQ || p->ent_scope > ULORL_ENT_SUPPLIED) return ULORL_ERR_INVALID_ARG;
+  if (p->loss_norm < ULORL_NORM_TOKENS || p->loss_norm > ULORL_NORM_SEQUENCE || p->norm_seqs < 0)
+    return ULORL_ERR_INVALID_ARG;
   if (p->kernel_path < ULORL_PATH_AUTO || p->kernel_path > ULORL_PATH_TENSOR) return ULORL_ERR_INVALID_ARG;
   if (p->kernel_path == ULORL_PATH_TENSOR && p->dtype != ULORL_BF16) return ULORL_ERR_UNSUPPORTED;
   if (!(p->inv_temperature > 0.f) || !std::isfinite(p->inv_temperature)) return ULORL_ERR_INVALID_ARG;
@@ -296,13 +298,15 @@ static DecideConsts make_decide_consts(const ulorl_params_t* p) {
   c.sigma = p->entropy_target;
   c.eps_lo = (double)p->clip_eps_low;
   c.eps_hi = (double)p->clip_eps_high;
-  const double N = p->norm_tokens > 0 ? (double)p->norm_tokens : (double)p->T;
+  double N = p->norm_tokens > 0 ? (double)p->norm_tokens : (double)p->T;
+  if (p->loss_norm == ULORL_NORM_SEQUENCE) N = p->norm_seqs > 0 ? (double)p->norm_seqs : (double)p->num_seqs;
   c.inv_N = N > 0 ? 1.0 / N : 0.0;
   c.is_mode = p->is_mode;
   c.mpt_mode = p->mpt_mode;
   c.ent_scope = p->ent_scope;
   c.adv_per_token = p->adv_per_token;
   c.current_version = p->current_version;
+  c.loss_norm = p->loss_norm;
   return c;
 }
 

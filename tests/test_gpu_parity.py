@@ -60,6 +60,8 @@ def check_against_oracle(batch, gp, op, grad_loss=None, check_grads=True):
     assert np.allclose(g[same], ref["grad_coef"][same], rtol=2 * TOL_LOGP, atol=1e-12)
     loss = float(out.loss.cpu()[0])
     N = float(op.norm_tokens) if op.norm_tokens > 0 else float(batch.workload.T)
+    if op.loss_norm == "sequence":                                        # a token weighs at most 1/G there
+        N = float(op.norm_seqs) if op.norm_seqs > 0 else float(S)
     flip_slack = float(np.abs(ref["surrogate"][differ]).sum()) / N        # what flipped tokens can move
     assert abs(loss - ref["loss"]) <= TOL_LOSS * max(abs(ref["loss"]), 1e-3) + flip_slack
     if not differ.any():
@@ -524,3 +526,22 @@ def test_token_range_split_with_entropy_exchange_matches_the_unsplit_batch():
     assert abs(loss - float(full.loss.cpu()[0])) <= 1e-5 * max(1e-3, abs(loss))
     assert torch.equal(dH, dH_full)                            # rows are independent of the split
     assert rel_l2(dW.cpu().numpy(), dW_full.cpu().numpy()) <= 1e-4
+
+
+@pytest.mark.parametrize("path,norm_seqs", [("tensor", 0), ("simt", 9)])
+def test_per_sample_normalisation_matches_the_oracle(path, norm_seqs):
+    """Eq. 5's (1/G) sum_i (1/|o_i|) weights instead of Eq. 10's 1/N: loss, coefficients and both gradients
+    against the oracle on ragged sequence lengths; the decisions are those of the token-normalised run."""
+    wl = synth.WORKLOADS["small"].scaled(T=700, S=5, H=328, V=3001, lengths="lognormal:100:400",
+                                         segment_len=64, planted=0.3, beta_planted=(80.0, 160.0),
+                                         mpt_mode="dynamic", entropy_target=6.0)
+    batch = synth.make_batch(wl, seed=5)
+    gp, op = both_params(batch, kernel_path=path, loss_norm="sequence", norm_seqs=norm_seqs)
+    out, ref = check_against_oracle(batch, gp, op)
+    gp_t, _ = both_params(batch, kernel_path=path)
+    out_t, _, _ = gpu_fwd_bwd(batch, gp_t)
+    assert torch.equal(out.flags, out_t.flags)
+    lens = np.diff(batch.seq_offsets.numpy())
+    G = norm_seqs if norm_seqs else wl.S
+    scale = np.repeat(wl.T / (G * lens.astype(np.float64)), lens)          # (1/(G|o_i|)) / (1/T)
+    assert np.allclose(out.grad_coef.cpu().numpy(), out_t.grad_coef.cpu().numpy() * scale, rtol=1e-6, atol=1e-12)

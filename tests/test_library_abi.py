@@ -34,7 +34,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_struct_sizes_match_header(lib):
     # 9 int32 + 5 float + (pad) int64 + 5 int32 (+ pad)
-    assert ctypes.sizeof(B.CParams) == 88
+    assert ctypes.sizeof(B.CParams) == 96
     assert ctypes.sizeof(B.CStats) == 4 * (2 + 6 + 3 * 16 + 4)
 
 
