@@ -104,3 +104,18 @@ def exchange_sequence_entropy(piece_mean: torch.Tensor, piece_tokens: torch.Tens
     if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
         dist.all_reduce(acc)
     return sequence_entropy_from_partials(acc, ids)
+
+
+def step_entropy_gate(call_mean_entropy: Sequence[float], call_tokens: Sequence[int], device=None) -> float:
+    """The gate entropy of Eq. 10 read as the entropy of the model over one optimiser step: the
+    token-weighted mean of the per-call mean entropies (the forward call's mean_entropy statistic) of all
+    micro-batches of this rank and, when a process group is up, of all ranks.  Every call of the step then
+    takes it for each of its sequences (ent_scope = supplied), so that micro-batching and sharding do not
+    change which tokens are masked."""
+    acc = torch.zeros(2, dtype=torch.float64, device=device)
+    for m, n in zip(call_mean_entropy, call_tokens):
+        acc[0] += float(m) * int(n)
+        acc[1] += int(n)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(acc)
+    return float(acc[0] / acc[1]) if float(acc[1]) > 0 else 0.0
