@@ -119,6 +119,19 @@ __device__ __forceinline__ float ex2f(float x) {
   return y;
 }
 
+// raw[idx] for an index only known at run time, as a chain of predicated moves over registers.  Written
+// as a plain select loop the compiler turns it into an indexed read, which puts the whole chunk in
+// local memory: every accumulator then goes through a store and a load (128 bytes of stack per
+// thread), and the statistics kernel loses a sixth of its rate.
+__device__ __forceinline__ float pick_column(const uint32_t (&raw)[32], int idx) {
+  uint32_t v = 0u;
+#pragma unroll
+  for (int j = 0; j < 32; ++j)
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.s32 p, %1, %2;\n\t@p mov.b32 %0, %3;\n\t}"
+                 : "+r"(v) : "r"(idx), "r"(j), "r"(raw[j]));
+  return __uint_as_float(v);
+}
+
 // One 32-column chunk of a row folded into the running (m, s, u) with m the max of the raw
 // accumulators a, s = sum 2^(c2 (a - m)) and u = sum 2^(c2 (a - m)) (a - m).  Keeping u relative to the
 // max makes the entropy ln s - kappa u / s free of cancellation for sharply peaked rows, and the
@@ -490,10 +503,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             if (nvalid >= 32) stats_chunk<true>(raw, 32, c2, run_m, run_s, run_u);
             else stats_chunk<false>(raw, nvalid, c2, run_m, run_s, run_u);
             if (row_ok && y >= col0 && y < col0 + 32) {
-              float ay = 0.f;
-#pragma unroll
-              for (int j = 0; j < 32; ++j) ay = (j == y - col0) ? __uint_as_float(raw[j]) : ay;
-              args.acc_y[grow] = ay;
+              args.acc_y[grow] = pick_column(raw, y - col0);
             }
           } else if (kMode == kModeDz) {
             uint32_t packed[16];
