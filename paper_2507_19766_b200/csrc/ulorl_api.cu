@@ -279,7 +279,7 @@ template <int kMode>
 static constexpr int acc_per_unit_pair() { return (kMode == kModeDHidden || kMode == kModeDW) ? 2 : 1; }
 static int grad_unit_cols() { return cta_group() == 2 ? 2 * kBN : kBN; }
 
-// mc is the output tensor map of the d_W kernel; the other kernels get any valid map and ignore it.
+// mc is the output tensor map of the dz and d_W kernels; the other kernels get any valid map and ignore it.
 template <int kMode>
 static int launch_umma(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const UmmaArgs& a,
                        cudaStream_t stream) {
@@ -364,6 +364,9 @@ struct StepHooks {
   int chunk_tokens = 0;
   std::function<int(int, int)> before_stats_chunk;    // (first token, tokens) -> status
   std::function<int(int, int)> after_dhidden_panel;   // (first token, tokens) -> status; dense backward only
+  // Tensor path: when set, the last panel computes d_W before d_hidden and in slabs of vocabulary rows,
+  // and this is called after each slab (first row, rows): those rows of d_W are final from then on.
+  std::function<int(int, int)> after_dw_slab;
 };
 
 }  // namespace ulorl
@@ -581,6 +584,9 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
     CUtensorMap map_dw_out;   // d_W as the target of 128-row x 32-column float tiles
     st = make_map(&map_dw_out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, d_W, (uint64_t)V, (uint64_t)H, (uint64_t)H, 32, kBM);
     if (st != ULORL_OK) return st;
+    CUtensorMap map_dz_out;   // the dz panel (all its rows) as the target of 128-row x 64-column bf16 tiles
+    st = make_map_bf16(&map_dz_out, dz, (uint64_t)pl.panel_tokens, (uint64_t)pl.dz_ld, (uint64_t)pl.dz_ld, 64, kBM);
+    if (st != ULORL_OK) return st;
     for (int t0 = 0, panel = 0; t0 < T; t0 += pl.panel_tokens, ++panel) {
       const int rows = (T - t0) < pl.panel_tokens ? (T - t0) : pl.panel_tokens;
       // dz panel: recompute logits, softmax minus one-hot scaled by the token's coefficient
@@ -594,10 +600,10 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
         a.row0 = t0;
         a.kappa = kappa;
         a.targets = targets; a.lse = lse; a.grad_coef = grad_coef; a.grad_loss = grad_loss;
-        a.dz = dz; a.dz_ld = pl.dz_ld; a.dz_cols = (int)pl.dz_ld;
+        a.dz_cols = (int)pl.dz_ld;
         a.dyn_rows = n_active; a.dyn_base = t0;
         a.status = status;
-        st = launch_umma<kModeDz>(map_hidden_k, map_w_k, map_w_k, a, stream);
+        st = launch_umma<kModeDz>(map_hidden_k, map_w_k, map_dz_out, a, stream);
         if (st != ULORL_OK) return st;
       }
       CUtensorMap map_dz_k, map_dz_mn;
@@ -606,7 +612,7 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
       st = make_map_bf16(&map_dz_mn, dz, (uint64_t)rows, (uint64_t)pl.dz_ld, (uint64_t)pl.dz_ld, 64, kBK);
       if (st != ULORL_OK) return st;
       // d_hidden[t0 + m, h] = sum_v dz[m, v] W[v, h]
-      {
+      auto run_d_hidden = [&]() -> int {
         UmmaArgs a{};
         a.M = rows; a.N = H; a.K = V;
         a.m_tiles = (rows + tile_m - 1) / tile_m;
@@ -617,27 +623,49 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
         a.out_ld = (size_t)H;
         a.dyn_rows = n_active; a.dyn_base = t0;
         a.status = status;
-        st = launch_umma<kModeDHidden>(map_dz_k, map_w_mn, map_w_mn, a, stream);
-        if (st != ULORL_OK) return st;
-        if (hooks && hooks->after_dhidden_panel && !pl.compact) {
-          st = hooks->after_dhidden_panel(t0, rows);
-          if (st != ULORL_OK) return st;
-        }
-      }
-      // d_W[v, h] (+)= sum_m dz[m, v] hidden[t0 + m, h]
-      {
+        int rc = launch_umma<kModeDHidden>(map_dz_k, map_w_mn, map_w_mn, a, stream);
+        if (rc != ULORL_OK) return rc;
+        if (hooks && hooks->after_dhidden_panel && !pl.compact) return hooks->after_dhidden_panel(t0, rows);
+        return ULORL_OK;
+      };
+      // d_W[v, h] (+)= sum_m dz[m, v] hidden[t0 + m, h] for the vocabulary rows [v0, v0 + v_rows)
+      auto run_d_W = [&](int v0, int v_rows) -> int {
         UmmaArgs a{};
-        a.M = V; a.N = H; a.K = rows;
-        a.m_tiles = (V + tile_m - 1) / tile_m;
+        a.M = v_rows; a.N = H; a.K = rows;
+        a.m_tiles = (v_rows + tile_m - 1) / tile_m;
         a.n_tiles = (H + grad_unit_cols() - 1) / grad_unit_cols();
         a.group_m = kGradRasterGroup;
+        a.a_mn0 = v0;
         a.b_k0 = t0;
+        a.row0 = v0;
         a.d_W = d_W;
         a.out_ld = (size_t)H;
         a.accumulate = (panel > 0 || params->dw_accumulate || pl.compact) ? 1 : 0;
         a.dyn_rows = n_active; a.dyn_base = t0;
         a.status = status;
-        st = launch_umma<kModeDW>(map_dz_mn, map_hidden_mn, map_dw_out, a, stream);
+        return launch_umma<kModeDW>(map_dz_mn, map_hidden_mn, map_dw_out, a, stream);
+      };
+      const bool last_panel = t0 + pl.panel_tokens >= T;
+      if (last_panel && hooks && hooks->after_dw_slab) {
+        // d_W is final slab by slab, so the caller can start moving it while the rest is computed; a slab
+        // is a whole number of waves of units (row tiles in multiples of the worker count), about eight
+        const int workers = kDesignSMs / cta_group();
+        const int v_tiles = (V + tile_m - 1) / tile_m;
+        const int slab_tiles = workers * ((v_tiles + 8 * workers - 1) / (8 * workers));
+        const int slab_rows = slab_tiles * tile_m;
+        for (int v0 = 0; v0 < V; v0 += slab_rows) {
+          const int v_rows = (V - v0) < slab_rows ? (V - v0) : slab_rows;
+          st = run_d_W(v0, v_rows);
+          if (st != ULORL_OK) return st;
+          st = hooks->after_dw_slab(v0, v_rows);
+          if (st != ULORL_OK) return st;
+        }
+        st = run_d_hidden();
+        if (st != ULORL_OK) return st;
+      } else {
+        st = run_d_hidden();
+        if (st != ULORL_OK) return st;
+        st = run_d_W(0, V);
         if (st != ULORL_OK) return st;
       }
     }
@@ -814,7 +842,15 @@ struct HostStepLayout {
 struct HostStepStreams {
   cudaStream_t in = nullptr, out = nullptr;
   cudaEvent_t start = nullptr, out_done = nullptr;
-  std::vector<cudaEvent_t> chunk_in, panel_out;
+  std::vector<cudaEvent_t> chunk_in, panel_out, slab_out;
+  cudaEvent_t slab_event(size_t i) {   // grows on demand; nullptr on failure
+    while (slab_out.size() <= i) {
+      cudaEvent_t e;
+      if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+      slab_out.push_back(e);
+    }
+    return slab_out[i];
+  }
   bool reserve(size_t n) {
     while (chunk_in.size() < n) {
       cudaEvent_t e0, e1;
@@ -935,6 +971,20 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
       return (int)ULORL_ERR_CUDA;
     return (int)ULORL_OK;
   };
+  // d_W rows go back slab by slab while the last panel is still being computed
+  size_t n_slabs = 0;
+  bool dw_by_slabs = false;
+  if (pl.tensor && h_d_W) {
+    hooks.after_dw_slab = [&](int v0, int v_rows) {
+      cudaEvent_t e = hs->slab_event(n_slabs++);
+      if (!e || !ok(cudaEventRecord(e, stream)) || !ok(cudaStreamWaitEvent(hs->out, e, 0)) ||
+          !ok(cudaMemcpyAsync(h_d_W + (size_t)v0 * H, a + L.d_W + (size_t)v0 * H * 4, (size_t)v_rows * H * 4,
+                              cudaMemcpyDeviceToHost, hs->out)))
+        return (int)ULORL_ERR_CUDA;
+      dw_by_slabs = true;
+      return (int)ULORL_OK;
+    };
+  }
   st = fwd_impl(params, a + L.hidden, a + L.W, reinterpret_cast<const int32_t*>(a + L.targets),
                 h_old_logp ? reinterpret_cast<const float*>(a + L.old_logp) : nullptr,
                 h_segment_version ? reinterpret_cast<const int32_t*>(a + L.segver) : nullptr,
@@ -960,7 +1010,7 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
   if (st != ULORL_OK) return st;
   // with compaction d_hidden is only final after the scatter at the end of the backward
   if (pl.compact && !ok(d2h(h_d_hidden, L.d_hidden, T * row_bytes))) return ULORL_ERR_CUDA;
-  if (!ok(d2h(h_d_W, L.d_W, V * H * 4))) return ULORL_ERR_CUDA;
+  if (!dw_by_slabs && !ok(d2h(h_d_W, L.d_W, V * H * 4))) return ULORL_ERR_CUDA;
   // the caller's stream is done only when the outbound copies are
   if (!ok(cudaEventRecord(hs->out_done, hs->out)) || !ok(cudaStreamWaitEvent(stream, hs->out_done, 0))) return ULORL_ERR_CUDA;
   return ULORL_OK;

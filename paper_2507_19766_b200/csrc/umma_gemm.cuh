@@ -81,9 +81,8 @@ struct UmmaArgs {
   float4* partials;         // kModeStats: [n_split][T_total]
   float* acc_y;             // kModeStats: raw accumulator at the target column, [T_total]
   int T_total;
-  __nv_bfloat16* dz;        // kModeDz: panel [rows][dz_ld]
-  size_t dz_ld;
-  int dz_cols;              // kModeDz: columns to write per row (>= N, zero beyond N)
+  int dz_cols;              // kModeDz: columns of the panel written per row (>= N, zero beyond N); the panel
+                            // itself is reached through the kernel's third tensor map
   __nv_bfloat16* d_hidden;  // kModeDHidden: [T][out_ld]
   float* d_W;               // kModeDW: [V][out_ld]
   size_t out_ld;
@@ -172,24 +171,34 @@ __device__ __forceinline__ void stats_chunk(const uint32_t (&raw)[32], int nvali
   run_u += u0 + u1;
 }
 
-// One 32-column chunk of dz = coef * (onehot - 2^(c2 a - lse2)), packed to bf16 pairs; columns at or
-// beyond nvalid give zero.  y_rel is the target column relative to the chunk (any value if outside).
+// One 32-column chunk of dz without its one-hot term: -coef * softmax = -sgn(coef) 2^(c2 a + k_row) with
+// k_row = log2|coef| - lse log2(e), so an element costs one fused multiply-add and one exponential; the sign
+// is applied to the packed bf16 pairs (sign_mask = 0x80008000 for coef > 0, else 0).  Columns at or beyond
+// nvalid give zero, and so does a row with coef = 0 (k_row = -inf).
 template <bool kFull>
-__device__ __forceinline__ void dz_chunk(const uint32_t (&raw)[32], int nvalid, int y_rel, float coef, float c2,
-                                         float lse2, uint32_t (&packed)[16]) {
+__device__ __forceinline__ void dz_chunk(const uint32_t (&raw)[32], int nvalid, float c2, float k_row,
+                                         uint32_t sign_mask, uint32_t* packed) {
 #pragma unroll
   for (int j = 0; j < 32; j += 2) {
-    float v0 = 0.f, v1 = 0.f;
-    if (kFull || j < nvalid) {
-      const float p = ex2f(fmaf(__uint_as_float(raw[j]), c2, -lse2));
-      v0 = coef * ((j == y_rel ? 1.f : 0.f) - p);
-    }
-    if (kFull || j + 1 < nvalid) {
-      const float p = ex2f(fmaf(__uint_as_float(raw[j + 1]), c2, -lse2));
-      v1 = coef * ((j + 1 == y_rel ? 1.f : 0.f) - p);
-    }
-    __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
-    packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h);
+    float e0 = 0.f, e1 = 0.f;
+    if (kFull || j < nvalid) e0 = ex2f(fmaf(__uint_as_float(raw[j]), c2, k_row));
+    if (kFull || j + 1 < nvalid) e1 = ex2f(fmaf(__uint_as_float(raw[j + 1]), c2, k_row));
+    __nv_bfloat162 h = __floats2bfloat162_rn(e0, e1);
+    packed[j >> 1] = *reinterpret_cast<uint32_t*>(&h) ^ sign_mask;
+  }
+}
+
+// packed[idx >> 1] with its half (idx & 1) replaced by the bf16 `half_bits`, for an index only known at run
+// time; predicated moves over registers for the same reason as pick_column.
+__device__ __forceinline__ void put_bf16(uint32_t (&packed)[32], int idx, uint32_t half_bits) {
+  const int word = idx >> 1;
+  const uint32_t keep = (idx & 1) ? 0x0000FFFFu : 0xFFFF0000u;
+  const uint32_t ins = (idx & 1) ? (half_bits << 16) : half_bits;
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    const uint32_t cand = (packed[j] & keep) | ins;
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.s32 p, %1, %2;\n\t@p mov.b32 %0, %3;\n\t}"
+                 : "+r"(packed[j]) : "r"(word), "r"(j), "r"(cand));
   }
 }
 
@@ -474,11 +483,15 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           }
         }
       }
+      float k_row = -INFINITY;                          // kModeDz: log2|coef| - lse log2(e); -inf gives a zero row
+      uint32_t sign_mask = 0u;
       if (kMode == kModeDz) {
         if (row_ok) {
           const float gl = args.grad_loss ? *args.grad_loss : 1.f;
           coef = args.kappa * gl * args.grad_coef[grow];
           lse2 = args.lse[grow] * 1.4426950408889634f;
+          if (coef != 0.f) k_row = log2f(fabsf(coef)) - lse2;
+          sign_mask = coef > 0.f ? 0x80008000u : 0u;
         }
       }
 
@@ -489,12 +502,57 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         if (!mbar_wait_bounded<true>(smem_u32(&bar_tmem_full[buf]), buf_phase, abort_p, kWaitLimitCycles)) goto role_done;
         tc_fence_after_sync();
         const uint32_t taddr = tmem_base + buf * kUnitN + ((uint32_t)(quarter * 32) << 16);
+        if (kMode == kModeDz) {
+          // 64 columns (one 128-byte row of bf16) at a time: two accumulator chunks -> packed registers ->
+          // swizzled staging tile in shared memory -> one TMA store of 128 rows x 128 bytes, so that the
+          // panel is written in whole lines by the copy engine instead of 16 bytes a thread
+          const int tile_row = (m_tile * kCta + cta_rank) * kBM;
+          const bool issuer = (threadIdx.x == 64);             // first thread of the epilogue warps
 #pragma unroll 1
-        for (int c = 0; c < kUnitN / 32; ++c) {
+          for (int g = 0; g < kUnitN / 64; ++g) {
+            const int col0 = col_base + g * 64;
+            if (col0 >= args.dz_cols) break;
+            uint32_t raw0[32], raw1[32];
+            tmem_ld_32x32(taddr + g * 64, raw0);
+            tmem_ld_32x32(taddr + g * 64 + 32, raw1);
+            tmem_ld_wait();
+            uint32_t packed[32];
+            const int nv0 = args.N - col0, nv1 = args.N - col0 - 32;
+            if (nv0 >= 32) dz_chunk<true>(raw0, 32, c2, k_row, sign_mask, packed);
+            else dz_chunk<false>(raw0, nv0, c2, k_row, sign_mask, packed);
+            if (nv1 >= 32) dz_chunk<true>(raw1, 32, c2, k_row, sign_mask, packed + 16);
+            else dz_chunk<false>(raw1, nv1, c2, k_row, sign_mask, packed + 16);
+            if (row_ok && y >= col0 && y < col0 + 64) {        // the one-hot term: coef (1 - p_y) at the target column
+              const int idx = y - col0;
+              const float ay = idx < 32 ? pick_column(raw0, idx) : pick_column(raw1, idx - 32);
+              const float vy = coef * (1.f - ex2f(fmaf(ay, c2, -lse2)));
+              const __nv_bfloat16 hv = __float2bfloat16_rn(vy);
+              put_bf16(packed, idx, (uint32_t)(*reinterpret_cast<const uint16_t*>(&hv)));
+            }
+            const uint32_t out_buf = smem_base + kStagesT * kStageBytesCta + (uint32_t)(g & 1) * kOutStageBytes;
+            if (issuer) bulk_wait_read_le1();                  // the copy that last read this staging tile is done with it
+            epilogue_bar_sync();
+            const uint32_t row_addr = out_buf + (uint32_t)row_in_tile * 128u;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const uint32_t dst = row_addr + ((uint32_t)(q ^ (row_in_tile & 7)) << 4);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(packed[4 * q]), "r"(packed[4 * q + 1]),
+                           "r"(packed[4 * q + 2]), "r"(packed[4 * q + 3])
+                           : "memory");
+            }
+            fence_async_proxy();
+            epilogue_bar_sync();
+            if (issuer) {
+              tma_store_2d(&map_c, out_buf, col0, tile_row);   // rows past the panel's capacity are clipped
+              bulk_commit_group();
+            }
+          }
+        }
+#pragma unroll 1
+        for (int c = 0; kMode != kModeDz && c < kUnitN / 32; ++c) {
           const int col0 = col_base + c * 32;
-          if (kMode != kModeDz && col0 >= args.N) break;       // whole chunk beyond the valid columns
-          if (kMode == kModeDz && col0 >= args.dz_cols) break;
-          const int nvalid = min(32, args.N - col0);           // may be <= 0 only in kModeDz padding
+          if (col0 >= args.N) break;                           // whole chunk beyond the valid columns
+          const int nvalid = min(32, args.N - col0);
           uint32_t raw[32];
           tmem_ld_32x32(taddr + c * 32, raw);
           tmem_ld_wait();
@@ -504,21 +562,6 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             else stats_chunk<false>(raw, nvalid, c2, run_m, run_s, run_u);
             if (row_ok && y >= col0 && y < col0 + 32) {
               args.acc_y[grow] = pick_column(raw, y - col0);
-            }
-          } else if (kMode == kModeDz) {
-            uint32_t packed[16];
-            if (nvalid >= 32) dz_chunk<true>(raw, 32, y - col0, coef, c2, lse2, packed);
-            else dz_chunk<false>(raw, nvalid, y - col0, coef, c2, lse2, packed);
-            if (!row_ok) {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) packed[j] = 0u;   // rows past M of a written tile read as zero later
-            }
-            {
-              uint4* dst = reinterpret_cast<uint4*>(args.dz + (size_t)row * args.dz_ld + col0);
-              const int ncols = min(32, args.dz_cols - col0);     // multiple of 8
-#pragma unroll
-              for (int q = 0; q < 4; ++q)
-                if (q * 8 < ncols) dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
             }
           } else if (kMode == kModeDHidden) {
             if (row_ok) {
@@ -573,7 +616,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   }
 
 role_done:
-  if (kMode == kModeDW && threadIdx.x == 64) bulk_wait_all();   // the tile copies have left shared memory and landed
+  if ((kMode == kModeDW || kMode == kModeDz) && threadIdx.x == 64) bulk_wait_all();   // the tile copies have left shared memory and landed
   if (*abort_p && lane == 0) atomicOr(args.status, kStatusTimeout);
   tc_fence_before_sync();
   __syncthreads();
