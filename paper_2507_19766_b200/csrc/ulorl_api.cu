@@ -17,6 +17,7 @@
 namespace ulorl {
 
 static std::atomic<long long> g_launches{0};
+constexpr size_t kStatsHiddenBudget = 40u << 20;   // live hidden tiles of the statistics kernel that L2 keeps beside W
 constexpr int kDesignSMs = 148;           // the plan (splits, workspace) is sized for a B200
 constexpr int kDefaultPanelTensor = 16384;       // single-CTA kernels
 constexpr int kDefaultPanelPair = 18944;         // CTA pairs: 74 pairs x 256 tokens, whole waves of d_hidden units
@@ -89,11 +90,19 @@ static Plan make_plan(const ulorl_params_t* p) {
   want = want > kMaxSplits ? kMaxSplits : want;
   want = want > n_tiles ? n_tiles : want;
   if (pl.tensor && m_tiles > 0) {
-    // persistent kernel: units = row tiles x splits are dealt round-robin to the workers, so the time is
-    // (waves of units) x (vocabulary tiles per split); take the split count from `want` up that wastes least
+    // Units (row tile, split) are dealt round-robin, splits fastest, to the persistent workers: at any time
+    // workers / splits row tiles are live, each sweeping its splits' slices of W side by side.  Their hidden
+    // tiles are re-read from L2 for every vocabulary tile, so they must fit beside the W streams -- few
+    // splits would not do (at H = 2048 one split means 74 MB of live hidden tiles) -- while every further
+    // split is one more pass of all of W through HBM per wave and one more stream for L2 to hold.  So:
+    // the smallest count that keeps the live hidden tiles within kStatsHiddenBudget, then the best of the
+    // next few for wave quantisation (time = waves of units x vocabulary tiles per split).
+    const size_t live_bytes = (size_t)workers * (size_t)tile_m * (size_t)p->H * 2;
+    const int fit = (int)((live_bytes + kStatsHiddenBudget - 1) / kStatsHiddenBudget);
+    if (fit > want) want = fit > n_tiles ? n_tiles : (fit > kMaxSplits ? kMaxSplits : fit);
     long best_cost = -1;
     int best = want;
-    for (int s = want; s <= kMaxSplits && s <= n_tiles; ++s) {
+    for (int s = want; s <= kMaxSplits && s <= n_tiles && s <= want + 3; ++s) {
       const int tps = (n_tiles + s - 1) / s;
       const int s_eff = (n_tiles + tps - 1) / tps;
       const long waves = ((long)m_tiles * s_eff + workers - 1) / workers;
@@ -240,10 +249,12 @@ static int launch_umma_impl(const CUtensorMap& ma, const CUtensorMap& mb, const 
   if (units <= 0) return ULORL_OK;
   if (kMode != kModeStats && a.group_m <= 0) return ULORL_ERR_INVALID_ARG;
   // L2 policy of the tile loads: keep what is re-read for long (the hidden tile of the two logits
-  // kernels, the slices of W / of the hidden panel that every pair sweeps in the gradient kernels)
+  // kernels, the slices of W / of the hidden panel that every pair sweeps in the gradient kernels).
+  // The statistics kernel marks its W stream too: it starts in an L2 that the gradient kernels of the
+  // step before left full of evict-last lines, which unmarked loads cannot displace.
   UmmaArgs a2 = a;
   a2.l2_a = (kMode == kModeStats || kMode == kModeDz) ? ptx::kL2EvictLast : ptx::kL2Normal;
-  a2.l2_b = (kMode == kModeDHidden || kMode == kModeDW) ? ptx::kL2EvictLast : ptx::kL2Normal;
+  a2.l2_b = (kMode == kModeStats || kMode == kModeDHidden || kMode == kModeDW) ? ptx::kL2EvictLast : ptx::kL2Normal;
   const int max_workers = num_sms / kCta;
   const int workers = units < max_workers ? units : max_workers;
   cudaEvent_t e0 = nullptr, e1 = nullptr;
