@@ -32,7 +32,7 @@ NOMINAL_BF16_TFLOPS = 2250.0
 # DRAM bytes (read + write) per launch of each tensor-core kernel at the full ultra workload, from the ncu
 # capture summarised in profiles/launch_list_ultra_full_size.md.  They describe the kernels as they were at
 # that capture: set an entry to None when its kernel changes, until the counters are taken again.
-NCU_TRAFFIC_BYTES = {"ultra": {"stats": 14.699e9, "dz": 8.871e9, "d_hidden": 9.353e9, "d_W": 12.315e9}}
+NCU_TRAFFIC_BYTES = {"ultra": {"stats": 9.320e9, "dz": 8.847e9, "d_hidden": 12.524e9, "d_W": 13.737e9}}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
