@@ -18,6 +18,7 @@ namespace ulorl {
 
 static std::atomic<long long> g_launches{0};
 constexpr size_t kStatsHiddenBudget = 40u << 20;   // live hidden tiles of the statistics kernel that L2 keeps beside W
+constexpr int kMaxDevices = 64;            // per-device set-up tables
 constexpr int kDesignSMs = 148;           // the plan (splits, workspace) is sized for a B200
 constexpr int kDefaultPanelTensor = 16384;       // single-CTA kernels
 constexpr int kDefaultPanelPair = 18944;         // CTA pairs: 74 pairs x 256 tokens, whole waves of d_hidden units
@@ -232,19 +233,20 @@ static cudaEvent_t timing_event(int kind) {
 template <int kMode, int kCta, int kAcc>
 static int launch_umma_impl(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const UmmaArgs& a,
                             cudaStream_t stream) {
-  static bool configured = false;
-  static int num_sms = 0;
+  // the shared-memory opt-in is a property of the function on ONE device: set up once per device
+  static int sms_of_device[kMaxDevices] = {};
   constexpr size_t smem = PipeConfig<kCta, kAcc, KAtoms<kMode, kCta>::value>::smem_bytes;
-  if (!configured) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ULORL_ERR_CUDA;
+  if (sms_of_device[dev] == 0) {
     if (cudaFuncSetAttribute(umma_kernel<kMode, kCta, kAcc>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)
       return ULORL_ERR_CUDA;
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0)
-      return ULORL_ERR_CUDA;
-    configured = true;
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return ULORL_ERR_CUDA;
+    sms_of_device[dev] = n;
   }
+  const int num_sms = sms_of_device[dev];
   const int units = (kMode == kModeStats) ? a.m_tiles * a.n_split : a.m_tiles * a.n_tiles;
   if (units <= 0) return ULORL_OK;
   if (kMode != kModeStats && a.group_m <= 0) return ULORL_ERR_INVALID_ARG;
@@ -874,16 +876,20 @@ struct HostStepStreams {
     return true;
   }
 };
+// Streams and events belong to the device that was current when they were made: one set per device.
 HostStepStreams* host_step_streams() {
-  static HostStepStreams hs;
-  static bool ready = false;
-  if (!ready) {
+  static HostStepStreams per_device[kMaxDevices];
+  static bool ready[kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  HostStepStreams& hs = per_device[dev];
+  if (!ready[dev]) {
     if (cudaStreamCreateWithFlags(&hs.in, cudaStreamNonBlocking) != cudaSuccess ||
         cudaStreamCreateWithFlags(&hs.out, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&hs.start, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&hs.out_done, cudaEventDisableTiming) != cudaSuccess)
       return nullptr;
-    ready = true;
+    ready[dev] = true;
   }
   return &hs;
 }
