@@ -396,14 +396,14 @@ def test_compacted_backward_with_nothing_active_and_with_accumulation():
 
 
 # --------------------------------------------------------------------------- host-buffer step, timing aid, bad offsets
-@pytest.mark.parametrize("V,panel", [(2500, 0), (40000, 512)])
-def test_host_buffer_step_matches_device_calls(V, panel):
+@pytest.mark.parametrize("V,panel,compact", [(2500, 0, False), (40000, 512, False), (40000, 512, True)])
+def test_host_buffer_step_matches_device_calls(V, panel, compact):
     # the second case has two backward panels and a vocabulary of several d_W slabs: on the last panel the
     # host-buffer step computes d_W slab by slab, ahead of d_hidden, and copies each slab out as it is done
     wl = synth.WORKLOADS["small"].scaled(T=900, S=4, H=256, V=V, lengths="tiny", planted=0.3,
                                          beta_planted=(100.0, 200.0), mpt_mode="always")
     batch = synth.make_batch(wl, seed=41)
-    gp, _ = both_params(batch, bwd_panel_tokens=panel)
+    gp, _ = both_params(batch, bwd_panel_tokens=panel, compact_rows=compact)
     out, dH, dW = gpu_fwd_bwd(batch, gp)
     arena = torch.empty(B.host_step_arena_bytes(gp), dtype=torch.uint8, device=DEV)
     pin = lambda t: t.contiguous().pin_memory()
