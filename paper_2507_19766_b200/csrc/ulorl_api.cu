@@ -2,6 +2,7 @@
 // construction and kernel launches.  No allocation, no synchronisation (except
 // ulorl_check_status), no state between calls.
 #include <atomic>
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -101,16 +102,18 @@ static Plan make_plan(const ulorl_params_t* p) {
     const size_t live_bytes = (size_t)workers * (size_t)tile_m * (size_t)p->H * 2;
     const int fit = (int)((live_bytes + kStatsHiddenBudget - 1) / kStatsHiddenBudget);
     if (fit > want) want = fit > n_tiles ? n_tiles : (fit > kMaxSplits ? kMaxSplits : fit);
-    long best_cost = -1;
-    int best = want;
-    for (int s = want; s <= kMaxSplits && s <= n_tiles && s <= want + 3; ++s) {
+    auto cost_of = [&](int s) {
       const int tps = (n_tiles + s - 1) / s;
       const int s_eff = (n_tiles + tps - 1) / tps;
       const long waves = ((long)m_tiles * s_eff + workers - 1) / workers;
-      const long cost = waves * tps;
-      if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
-    }
-    want = best;
+      return waves * tps;
+    };
+    const int s_max = std::min(std::min(want + 3, kMaxSplits), n_tiles);
+    long best_cost = cost_of(want);
+    for (int s = want + 1; s <= s_max; ++s) best_cost = cost_of(s) < best_cost ? cost_of(s) : best_cost;
+    // the fewest splits within one percent of the best: a split more costs HBM passes over W, not time
+    for (int s = want; s <= s_max; ++s)
+      if (cost_of(s) * 100 <= best_cost * 101) { want = s; break; }
   }
   pl.tiles_per_split = (n_tiles + want - 1) / want;
   pl.n_split = (n_tiles + pl.tiles_per_split - 1) / pl.tiles_per_split;
