@@ -11,8 +11,18 @@
  *
  * Conventions
  *  - Every pointer except `params` is DEVICE memory owned by the caller, row-major and
- *    contiguous.  The library allocates nothing, frees nothing and keeps no state
- *    between calls.
+ *    contiguous.  The library allocates and frees no device memory; results depend only on
+ *    the arguments of the call.
+ *  - State kept by the library (process lifetime, created on first use under one internal
+ *    mutex, so first calls from several host threads are safe): per device, the shared-memory
+ *    opt-in of each kernel, the multiprocessor count, the device address of the built-in
+ *    scratch of ulorl_token_loss_decide_static, and the two copy streams with their events of
+ *    ulorl_token_loss_step_host; per process, the driver entry point that encodes tensor
+ *    maps, the launch counter and the events of ulorl_kernel_timing_*.  No environment
+ *    variable is read.
+ *  - Every path is deterministic: no floating-point atomics; reductions over tokens run in a
+ *    fixed order (d_W: one reduce-add per element and panel, panels in order), so equal
+ *    inputs give bit-identical outputs on equal hardware.
  *  - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*) and never
  *    synchronise.  `loss` and `stats` stay on the device.
  *  - The return value is the host-side validation / launch status.  Device-side problems
@@ -47,7 +57,10 @@ typedef enum { ULORL_F32 = 0, ULORL_BF16 = 1 } ulorl_dtype_t;
 typedef enum { ULORL_IS_SAIS = 0, ULORL_IS_POIS = 1 } ulorl_is_mode_t;            /* Eq. 8 | Section 3.1.2 */
 typedef enum { ULORL_MPT_OFF = 0, ULORL_MPT_ALWAYS = 1, ULORL_MPT_DYNAMIC = 2 } ulorl_mpt_mode_t; /* Section 3.2 */
 typedef enum { ULORL_ENT_PER_SEQ = 0, ULORL_ENT_BATCH = 1, ULORL_ENT_SUPPLIED = 2 } ulorl_ent_scope_t;
-typedef enum { ULORL_PATH_AUTO = 0, ULORL_PATH_SIMT = 1, ULORL_PATH_TENSOR = 2 } ulorl_kernel_path_t;
+/* AUTO = TENSOR for bf16, SIMT for f32.  TENSOR: tcgen05 kernels on CTA pairs (one 256 x 256 MMA tile per
+ * pair).  TENSOR_1CTA: the same kernels with one CTA per 128 x 256 tile, kept as a cross-check. */
+typedef enum { ULORL_PATH_AUTO = 0, ULORL_PATH_SIMT = 1, ULORL_PATH_TENSOR = 2,
+               ULORL_PATH_TENSOR_1CTA = 3 } ulorl_kernel_path_t;
 
 /* bits of flags[t] */
 #define ULORL_FLAG_MASKED    1u  /* MPT and gate open: excluded from the objective (Eq. 10)   */

@@ -21,7 +21,7 @@ F32, BF16 = 0, 1
 IS_SAIS, IS_POIS = 0, 1
 MPT_OFF, MPT_ALWAYS, MPT_DYNAMIC = 0, 1, 2
 ENT_PER_SEQ, ENT_BATCH, ENT_SUPPLIED = 0, 1, 2
-PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
+PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_TENSOR_1CTA = 0, 1, 2, 3
 FLAG_MASKED, FLAG_CLIP_HIGH, FLAG_CLIP_LOW, FLAG_MPT = 1, 2, 4, 8
 N_STALENESS = 16
 
@@ -29,7 +29,7 @@ _IS = {"sais": IS_SAIS, "pois": IS_POIS}
 _MPT = {"off": MPT_OFF, "always": MPT_ALWAYS, "dynamic": MPT_DYNAMIC}
 _ENT = {"per_seq": ENT_PER_SEQ, "batch": ENT_BATCH, "supplied": ENT_SUPPLIED}
 _NORM = {"tokens": 0, "sequence": 1}
-_PATH = {"auto": PATH_AUTO, "simt": PATH_SIMT, "tensor": PATH_TENSOR}
+_PATH = {"auto": PATH_AUTO, "simt": PATH_SIMT, "tensor": PATH_TENSOR, "tensor_1cta": PATH_TENSOR_1CTA}
 
 
 class UlorlError(RuntimeError):

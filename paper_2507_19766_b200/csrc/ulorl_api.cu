@@ -1,6 +1,7 @@
 // C ABI of the UloRL token-loss library: argument validation, workspace carve-up, tensor-map
-// construction and kernel launches.  No allocation, no synchronisation (except
-// ulorl_check_status), no state between calls.
+// construction and kernel launches.  No device allocation and no synchronisation (except
+// ulorl_check_status and ulorl_kernel_timing_end).  What the process keeps between calls is listed
+// in ulorl.h ("State kept by the library") and is created under g_setup_mutex.
 #include <atomic>
 #include <algorithm>
 #include <cmath>
@@ -8,6 +9,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <functional>
+#include <mutex>
 #include <vector>
 
 #include "common.cuh"
@@ -20,26 +22,42 @@ namespace ulorl {
 static std::atomic<long long> g_launches{0};
 constexpr size_t kStatsHiddenBudget = 40u << 20;   // live hidden tiles of the statistics kernel that L2 keeps beside W
 constexpr int kMaxDevices = 64;            // per-device set-up tables
-constexpr int kDesignSMs = 148;           // the plan (splits, workspace) is sized for a B200
+constexpr int kFallbackSMs = 148;         // B200; used for the plan when no device can be asked
 constexpr int kDefaultPanelTensor = 16384;       // single-CTA kernels
-constexpr int kDefaultPanelPair = 18944;         // CTA pairs: 74 pairs x 256 tokens, whole waves of d_hidden units
 constexpr int kDefaultPanelSimt = 1024;
 constexpr int kRasterGroup = 16;          // dz: row tiles per raster group (m fastest inside a group)
 constexpr int kGradRasterGroup = 1;       // d_hidden, d_W: column blocks of one row tile run side by side, so its A stream is read once
 
-// CTAs per tcgen05.mma: 2 (a CTA pair per 256 x 256 tile, the default) or 1.  The environment
-// variable ULORL_CTA_GROUP=1 selects the single-CTA kernels (read once per process).
-static int cta_group() {
-  static int value = 0;
-  if (value == 0) {
-    const char* e = std::getenv("ULORL_CTA_GROUP");
-    value = (e && e[0] == '1') ? 1 : 2;
+// Everything the library creates lazily and keeps (per-device tables, events, streams, the driver
+// entry point) is created and looked up under this one mutex, so that first calls from several host
+// threads do not race.
+static std::mutex g_setup_mutex;
+
+// Multiprocessor count of the current device (asked once per device); kFallbackSMs when there is
+// no device to ask, so that ulorl_workspace_bytes stays usable on a host without a GPU.
+static int device_sm_count() {
+  static int sms[kMaxDevices] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    (void)cudaGetLastError();
+    return kFallbackSMs;
   }
-  return value;
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
+  if (sms[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+      (void)cudaGetLastError();
+      return kFallbackSMs;
+    }
+    sms[dev] = n;
+  }
+  return sms[dev];
 }
 
 struct Plan {
   bool tensor;            // tensor-core path (bf16) or SIMT path
+  int cta;                // CTAs per tcgen05.mma: 2 (a CTA pair per 256 x 256 tile) or 1 (ULORL_PATH_TENSOR_1CTA)
+  int sms;                // multiprocessors the persistent kernels are spread over
   int n_split, tiles_per_split;
   int panel_tokens;
   size_t dz_ld;           // leading dimension of the dz panel (elements)
@@ -67,8 +85,9 @@ static int validate_params(const ulorl_params_t* p) {
   if (p->ent_scope < ULORL_ENT_PER_SEQ || p->ent_scope > ULORL_ENT_SUPPLIED) return ULORL_ERR_INVALID_ARG;
   if (p->loss_norm < ULORL_NORM_TOKENS || p->loss_norm > ULORL_NORM_SEQUENCE || p->norm_seqs < 0)
     return ULORL_ERR_INVALID_ARG;
-  if (p->kernel_path < ULORL_PATH_AUTO || p->kernel_path > ULORL_PATH_TENSOR) return ULORL_ERR_INVALID_ARG;
-  if (p->kernel_path == ULORL_PATH_TENSOR && p->dtype != ULORL_BF16) return ULORL_ERR_UNSUPPORTED;
+  if (p->kernel_path < ULORL_PATH_AUTO || p->kernel_path > ULORL_PATH_TENSOR_1CTA) return ULORL_ERR_INVALID_ARG;
+  if ((p->kernel_path == ULORL_PATH_TENSOR || p->kernel_path == ULORL_PATH_TENSOR_1CTA) && p->dtype != ULORL_BF16)
+    return ULORL_ERR_UNSUPPORTED;
   if (!(p->inv_temperature > 0.f) || !std::isfinite(p->inv_temperature)) return ULORL_ERR_INVALID_ARG;
   if (!(p->clip_eps_low >= 0.f) || !(p->clip_eps_high >= 0.f) || p->clip_eps_low > 1.f) return ULORL_ERR_INVALID_ARG;
   if (!(p->mpt_tau > 0.f) || p->mpt_tau > 1.f) return ULORL_ERR_INVALID_ARG;
@@ -81,10 +100,12 @@ static int validate_params(const ulorl_params_t* p) {
 static Plan make_plan(const ulorl_params_t* p) {
   Plan pl{};
   pl.tensor = use_tensor_path(p);
+  pl.cta = p->kernel_path == ULORL_PATH_TENSOR_1CTA ? 1 : 2;
+  pl.sms = device_sm_count();
   const int T = p->T, V = p->V;
-  const int tile_m = pl.tensor ? kBM * cta_group() : kSimtTile;
+  const int tile_m = pl.tensor ? kBM * pl.cta : kSimtTile;
   const int tile_n = pl.tensor ? kBN : kSimtTile;
-  const int workers = pl.tensor ? kDesignSMs / cta_group() : kDesignSMs;
+  const int workers = pl.tensor ? std::max(1, pl.sms / pl.cta) : pl.sms;
   const int m_tiles = (T + tile_m - 1) / tile_m;
   const int n_tiles = (V + tile_n - 1) / tile_n;
   int want = m_tiles > 0 ? (8 * workers + m_tiles - 1) / m_tiles : 1;
@@ -118,8 +139,8 @@ static Plan make_plan(const ulorl_params_t* p) {
   pl.tiles_per_split = (n_tiles + want - 1) / want;
   pl.n_split = (n_tiles + pl.tiles_per_split - 1) / pl.tiles_per_split;
   int panel = p->bwd_panel_tokens > 0 ? p->bwd_panel_tokens
-                                      : (pl.tensor ? (cta_group() == 2 ? kDefaultPanelPair : kDefaultPanelTensor) : kDefaultPanelSimt);
-  const int panel_unit = pl.tensor ? kBM * cta_group() : kBM;   // whole row tiles: the dz kernel zero-fills to the tile end
+                                      : (pl.tensor ? (pl.cta == 2 ? workers * kBM * 2 : kDefaultPanelTensor) : kDefaultPanelSimt);
+  const int panel_unit = pl.tensor ? kBM * pl.cta : kBM;   // whole row tiles: the dz kernel zero-fills to the tile end
   panel = (panel + panel_unit - 1) / panel_unit * panel_unit;
   const int t_round = (T + panel_unit - 1) / panel_unit * panel_unit;
   if (panel > t_round) panel = t_round;
@@ -178,6 +199,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 static EncodeTiledFn get_encode_fn() {
   static EncodeTiledFn fn = nullptr;
   static bool tried = false;
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
   if (!tried) {
     tried = true;
     void* ptr = nullptr;
@@ -217,7 +239,7 @@ static int make_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uint
 // Optional per-kernel timing of the tensor-core launches: when enabled, an event pair brackets
 // every launch on its stream, so durations are measured inside whatever region the caller times.
 struct KernelTiming {
-  bool enabled = false;
+  std::atomic<bool> enabled{false};
   std::vector<cudaEvent_t> ev[4];   // start/stop pairs per kernel kind
   size_t used[4] = {0, 0, 0, 0};
 };
@@ -225,6 +247,7 @@ static KernelTiming g_timing;
 
 static cudaEvent_t timing_event(int kind) {
   KernelTiming& t = g_timing;
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
   if (t.used[kind] == t.ev[kind].size()) {
     cudaEvent_t e;
     if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
@@ -235,21 +258,21 @@ static cudaEvent_t timing_event(int kind) {
 
 template <int kMode, int kCta, int kAcc>
 static int launch_umma_impl(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const UmmaArgs& a,
-                            cudaStream_t stream) {
+                            int num_sms, cudaStream_t stream) {
   // the shared-memory opt-in is a property of the function on ONE device: set up once per device
-  static int sms_of_device[kMaxDevices] = {};
+  static bool opted_in[kMaxDevices] = {};
   constexpr size_t smem = PipeConfig<kCta, kAcc, KAtoms<kMode, kCta>::value>::smem_bytes;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ULORL_ERR_CUDA;
-  if (sms_of_device[dev] == 0) {
-    if (cudaFuncSetAttribute(umma_kernel<kMode, kCta, kAcc>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-        cudaSuccess)
-      return ULORL_ERR_CUDA;
-    int n = 0;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return ULORL_ERR_CUDA;
-    sms_of_device[dev] = n;
+  {
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    if (!opted_in[dev]) {
+      if (cudaFuncSetAttribute(umma_kernel<kMode, kCta, kAcc>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)smem) != cudaSuccess)
+        return ULORL_ERR_CUDA;
+      opted_in[dev] = true;
+    }
   }
-  const int num_sms = sms_of_device[dev];
   const int units = (kMode == kModeStats) ? a.m_tiles * a.n_split : a.m_tiles * a.n_tiles;
   if (units <= 0) return ULORL_OK;
   if (kMode != kModeStats && a.group_m <= 0) return ULORL_ERR_INVALID_ARG;
@@ -263,7 +286,7 @@ static int launch_umma_impl(const CUtensorMap& ma, const CUtensorMap& mb, const 
   const int max_workers = num_sms / kCta;
   const int workers = units < max_workers ? units : max_workers;
   cudaEvent_t e0 = nullptr, e1 = nullptr;
-  if (g_timing.enabled) {
+  if (g_timing.enabled.load(std::memory_order_relaxed)) {
     e0 = timing_event(kMode);
     e1 = timing_event(kMode);
     if (e0 && e1) cudaEventRecord(e0, stream);
@@ -293,14 +316,14 @@ static int launch_umma_impl(const CUtensorMap& ma, const CUtensorMap& mb, const 
 // Accumulators per unit: the gradient contractions on CTA pairs use two (256 x 512 outputs a unit).
 template <int kMode>
 static constexpr int acc_per_unit_pair() { return (kMode == kModeDHidden || kMode == kModeDW) ? 2 : 1; }
-static int grad_unit_cols() { return cta_group() == 2 ? 2 * kBN : kBN; }
+static int grad_unit_cols(const Plan& pl) { return pl.cta == 2 ? 2 * kBN : kBN; }
 
 // mc is the output tensor map of the dz and d_W kernels; the other kernels get any valid map and ignore it.
 template <int kMode>
-static int launch_umma(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const UmmaArgs& a,
-                       cudaStream_t stream) {
-  return cta_group() == 2 ? launch_umma_impl<kMode, 2, acc_per_unit_pair<kMode>()>(ma, mb, mc, a, stream)
-                          : launch_umma_impl<kMode, 1, 1>(ma, mb, mc, a, stream);
+static int launch_umma(const Plan& pl, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc,
+                       const UmmaArgs& a, cudaStream_t stream) {
+  return pl.cta == 2 ? launch_umma_impl<kMode, 2, acc_per_unit_pair<kMode>()>(ma, mb, mc, a, pl.sms, stream)
+                     : launch_umma_impl<kMode, 1, 1>(ma, mb, mc, a, pl.sms, stream);
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -471,9 +494,9 @@ static int fwd_impl(const ulorl_params_t* params, const void* hidden, const void
     CUtensorMap map_a, map_b;
     st = make_map_bf16(&map_a, hidden, (uint64_t)T, (uint64_t)H, (uint64_t)H, kBK, kBM);
     if (st != ULORL_OK) return st;
-    st = make_map_bf16(&map_b, W, (uint64_t)V, (uint64_t)H, (uint64_t)H, kBK, kBN / cta_group());
+    st = make_map_bf16(&map_b, W, (uint64_t)V, (uint64_t)H, (uint64_t)H, kBK, kBN / pl.cta);
     if (st != ULORL_OK) return st;
-    const int tile_m = kBM * cta_group();
+    const int tile_m = kBM * pl.cta;
     int chunk = (hooks && hooks->chunk_tokens > 0) ? hooks->chunk_tokens : T;
     chunk = (chunk + tile_m - 1) / tile_m * tile_m;
     for (int t0 = 0; t0 < T; t0 += chunk) {
@@ -496,7 +519,7 @@ static int fwd_impl(const ulorl_params_t* params, const void* hidden, const void
       a.acc_y = acc_y;
       a.T_total = T;
       a.status = status;
-      st = launch_umma<kModeStats>(map_a, map_b, map_a, a, stream);
+      st = launch_umma<kModeStats>(pl, map_a, map_b, map_a, a, stream);
       if (st != ULORL_OK) return st;
     }
   } else {
@@ -555,7 +578,7 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
 
   if (pl.tensor) {
     __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(ws + pl.off_dz);
-    const int tile_m = kBM * cta_group();
+    const int tile_m = kBM * pl.cta;
     // With compaction the three contractions run on gathered copies of the active rows; how many
     // there are is only known on the device, so every launch is sized for the worst case and reads
     // the count itself.
@@ -591,7 +614,7 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
     CUtensorMap map_hidden_k, map_w_k, map_w_mn, map_hidden_mn;
     st = make_map_bf16(&map_hidden_k, hidden, hidden_rows, (uint64_t)H, (uint64_t)H, kBK, kBM);
     if (st != ULORL_OK) return st;
-    st = make_map_bf16(&map_w_k, W, (uint64_t)V, (uint64_t)H, (uint64_t)H, kBK, kBN / cta_group());
+    st = make_map_bf16(&map_w_k, W, (uint64_t)V, (uint64_t)H, (uint64_t)H, kBK, kBN / pl.cta);
     if (st != ULORL_OK) return st;
     st = make_map_bf16(&map_w_mn, W, (uint64_t)V, (uint64_t)H, (uint64_t)H, 64, kBK);
     if (st != ULORL_OK) return st;
@@ -619,7 +642,7 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
         a.dz_cols = (int)pl.dz_ld;
         a.dyn_rows = n_active; a.dyn_base = t0;
         a.status = status;
-        st = launch_umma<kModeDz>(map_hidden_k, map_w_k, map_dz_out, a, stream);
+        st = launch_umma<kModeDz>(pl, map_hidden_k, map_w_k, map_dz_out, a, stream);
         if (st != ULORL_OK) return st;
       }
       CUtensorMap map_dz_k, map_dz_mn;
@@ -632,14 +655,14 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
         UmmaArgs a{};
         a.M = rows; a.N = H; a.K = V;
         a.m_tiles = (rows + tile_m - 1) / tile_m;
-        a.n_tiles = (H + grad_unit_cols() - 1) / grad_unit_cols();
+        a.n_tiles = (H + grad_unit_cols(pl) - 1) / grad_unit_cols(pl);
         a.group_m = kGradRasterGroup;
         a.row0 = t0;
         a.d_hidden = static_cast<__nv_bfloat16*>(d_hidden_out);
         a.out_ld = (size_t)H;
         a.dyn_rows = n_active; a.dyn_base = t0;
         a.status = status;
-        int rc = launch_umma<kModeDHidden>(map_dz_k, map_w_mn, map_w_mn, a, stream);
+        int rc = launch_umma<kModeDHidden>(pl, map_dz_k, map_w_mn, map_w_mn, a, stream);
         if (rc != ULORL_OK) return rc;
         if (hooks && hooks->after_dhidden_panel && !pl.compact) return hooks->after_dhidden_panel(t0, rows);
         return ULORL_OK;
@@ -649,7 +672,7 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
         UmmaArgs a{};
         a.M = v_rows; a.N = H; a.K = rows;
         a.m_tiles = (v_rows + tile_m - 1) / tile_m;
-        a.n_tiles = (H + grad_unit_cols() - 1) / grad_unit_cols();
+        a.n_tiles = (H + grad_unit_cols(pl) - 1) / grad_unit_cols(pl);
         a.group_m = kGradRasterGroup;
         a.a_mn0 = v0;
         a.b_k0 = t0;
@@ -659,13 +682,13 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
         a.accumulate = (panel > 0 || params->dw_accumulate || pl.compact) ? 1 : 0;
         a.dyn_rows = n_active; a.dyn_base = t0;
         a.status = status;
-        return launch_umma<kModeDW>(map_dz_mn, map_hidden_mn, map_dw_out, a, stream);
+        return launch_umma<kModeDW>(pl, map_dz_mn, map_hidden_mn, map_dw_out, a, stream);
       };
       const bool last_panel = t0 + pl.panel_tokens >= T;
       if (last_panel && hooks && hooks->after_dw_slab) {
         // d_W is final slab by slab, so the caller can start moving it while the rest is computed; a slab
         // is a whole number of waves of units (row tiles in multiples of the worker count), about eight
-        const int workers = kDesignSMs / cta_group();
+        const int workers = std::max(1, pl.sms / pl.cta);
         const int v_tiles = (V + tile_m - 1) / tile_m;
         const int slab_tiles = workers * ((v_tiles + 8 * workers - 1) / (8 * workers));
         const int slab_rows = slab_tiles * tile_m;
@@ -762,6 +785,7 @@ static int static_scratch_address(uint8_t** out) {
   static uint8_t* cached[kMaxDevices] = {};
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ULORL_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
   if (!cached[dev]) {
     void* ptr = nullptr;
     const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
@@ -822,14 +846,16 @@ int ulorl_group_advantages(const float* rewards, int32_t num_responses, int32_t 
 }
 
 int ulorl_kernel_timing_begin(void) {
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
   for (int k = 0; k < 4; ++k) g_timing.used[k] = 0;
-  g_timing.enabled = true;
+  g_timing.enabled.store(true);
   return ULORL_OK;
 }
 
 int ulorl_kernel_timing_end(float* total_ms, int64_t* launches) {
-  g_timing.enabled = false;
+  g_timing.enabled.store(false);
   if (!total_ms || !launches) return ULORL_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
   for (int k = 0; k < 4; ++k) {
     double tot = 0.0;
     int64_t n = 0;
@@ -856,6 +882,7 @@ struct HostStepLayout {
 // Two copy streams and a few events, created on the first host-buffer step and kept: the inbound
 // copies run ahead of the forward, the outbound copies of d_hidden behind the backward.
 struct HostStepStreams {
+  std::mutex step_mutex;   // held while one host-buffer step is enqueued: the streams and events are shared
   cudaStream_t in = nullptr, out = nullptr;
   cudaEvent_t start = nullptr, out_done = nullptr;
   std::vector<cudaEvent_t> chunk_in, panel_out, slab_out;
@@ -886,6 +913,7 @@ HostStepStreams* host_step_streams() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
   HostStepStreams& hs = per_device[dev];
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
   if (!ready[dev]) {
     if (cudaStreamCreateWithFlags(&hs.in, cudaStreamNonBlocking) != cudaSuccess ||
         cudaStreamCreateWithFlags(&hs.out, cudaStreamNonBlocking) != cudaSuccess ||
@@ -949,6 +977,7 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
   const size_t T = (size_t)params->T, H = (size_t)params->H, V = (size_t)params->V, S = (size_t)params->num_seqs;
   HostStepStreams* hs = host_step_streams();
   if (!hs) return ULORL_ERR_CUDA;
+  std::lock_guard<std::mutex> step_lock(hs->step_mutex);
   const Plan pl = make_plan(params);
   const size_t row_bytes = H * L.elem;
   auto ok = [](cudaError_t e) { return e == cudaSuccess; };

@@ -455,6 +455,11 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const int row_in_tile = quarter * 32 + lane;
     const float c2 = args.kappa * 1.4426950408889634f;  // exp(kappa a) = 2^(c2 a)
     uint32_t acc_iter = 0;
+    // The dz and d_W epilogues alternate between two staging tiles and only ever wait until at most ONE
+    // tile copy is still reading shared memory, so the tile must be chosen by a count of the copies
+    // issued that runs across accumulators and units: a last column tile that ends after an odd number
+    // of copies would otherwise hand the next unit the tile whose copy is the one still in flight.
+    uint32_t stage_iter = 0;
     for (int unit = worker; unit < n_units; unit += n_workers) {
       int m_tile, n_begin, n_end, split = 0;
       if (kMode == kModeStats) {
@@ -499,7 +504,11 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const uint32_t buf = acc_iter % kBufs;
         const uint32_t buf_phase = (acc_iter / kBufs) & 1u;
         const int col_base = n_tile * kUnitN;
-        if (!mbar_wait_bounded<true>(smem_u32(&bar_tmem_full[buf]), buf_phase, abort_p, kWaitLimitCycles)) goto role_done;
+        // The give-up decision is taken by the 128 epilogue threads together: a thread that saw the wait
+        // complete while another saw the abort flag would otherwise go on alone to warp-wide tensor-memory
+        // loads and to the epilogue barrier, which the others never reach.
+        if (!epilogue_all(mbar_wait_bounded<true>(smem_u32(&bar_tmem_full[buf]), buf_phase, abort_p, kWaitLimitCycles)))
+          goto role_done;
         tc_fence_after_sync();
         const uint32_t taddr = tmem_base + buf * kUnitN + ((uint32_t)(quarter * 32) << 16);
         if (kMode == kModeDz) {
@@ -529,7 +538,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
               const __nv_bfloat16 hv = __float2bfloat16_rn(vy);
               put_bf16(packed, idx, (uint32_t)(*reinterpret_cast<const uint16_t*>(&hv)));
             }
-            const uint32_t out_buf = smem_base + kStagesT * kStageBytesCta + (uint32_t)(g & 1) * kOutStageBytes;
+            const uint32_t out_buf = smem_base + kStagesT * kStageBytesCta + (stage_iter++ & 1u) * kOutStageBytes;
             if (issuer) bulk_wait_read_le1();                  // the copy that last read this staging tile is done with it
             epilogue_bar_sync();
             const uint32_t row_addr = out_buf + (uint32_t)row_in_tile * 128u;
@@ -577,7 +586,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 if (q * 8 < nvalid) dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
             }
           } else {  // kModeDW: swizzled staging tile, then one TMA store (first panel) or reduce-add
-            const uint32_t out_buf = smem_base + kStagesT * kStageBytesCta + (uint32_t)(c & 1) * kOutStageBytes;
+            const uint32_t out_buf = smem_base + kStagesT * kStageBytesCta + (stage_iter++ & 1u) * kOutStageBytes;
             const bool issuer = (threadIdx.x == 64);             // first thread of the epilogue warps
             if (issuer) bulk_wait_read_le1();                    // the copy that last read this tile is done with it
             epilogue_bar_sync();

@@ -143,7 +143,7 @@ def test_tiny_planted_mask_fires(mpt_mode):
     assert ref["stats"]["n_mpt"] > 20
 
 
-@pytest.mark.parametrize("path", ["tensor", "simt"])
+@pytest.mark.parametrize("path", ["tensor", "tensor_1cta", "simt"])
 def test_bf16_mini_ragged(path):
     """bf16, several token tiles with a ragged tail, vocabulary not a multiple of any tile width,
     hidden size not a multiple of the 64-element pipeline stage, two backward panels."""
@@ -152,6 +152,20 @@ def test_bf16_mini_ragged(path):
                                          mpt_mode="dynamic", entropy_target=6.0)
     batch = synth.make_batch(wl, seed=5)
     gp, op = both_params(batch, kernel_path=path, bwd_panel_tokens=384)
+    check_against_oracle(batch, gp, op)
+
+
+@pytest.mark.parametrize("path", ["tensor", "tensor_1cta"])
+def test_odd_staging_tile_counts_across_units(path):
+    """The dz and d_W epilogues hand tiles to the copy engine through two alternating staging buffers.
+    Here the last column tile of a unit ends after an odd number of copies (ceil(V / 64) = 301 = 1 mod 4 for
+    dz, H / 32 = 11 chunks for d_W) and every persistent worker runs more than one unit (3 x 76 dz units,
+    76 d_W units on 74 or 148 workers), so a worker's next unit starts right behind an odd count."""
+    wl = synth.WORKLOADS["small"].scaled(T=600, S=4, H=352, V=19264, lengths="lognormal:100:300", segment_len=64,
+                                         planted=0.3, beta_planted=(80.0, 160.0), mpt_mode="dynamic",
+                                         entropy_target=6.0)
+    batch = synth.make_batch(wl, seed=51)
+    gp, op = both_params(batch, kernel_path=path, bwd_panel_tokens=512)
     check_against_oracle(batch, gp, op)
 
 
@@ -189,14 +203,19 @@ def test_tensor_path_matches_simt_path():
     wl = synth.WORKLOADS["small"].scaled(T=1000, S=3, H=512, V=5000, lengths="lognormal:300:600", segment_len=128)
     batch = synth.make_batch(wl, seed=21)
     res = {}
-    for path in ("tensor", "simt"):
+    for path in ("tensor", "tensor_1cta", "simt"):
         gp, _ = both_params(batch, kernel_path=path)
         res[path] = gpu_fwd_bwd(batch, gp)
-    a, b = res["tensor"], res["simt"]
-    assert (a[0].logp - b[0].logp).abs().max() <= 1e-4
-    assert (a[0].entropy - b[0].entropy).abs().max() <= 1e-4
-    assert rel_l2(a[1].float().cpu().numpy(), b[1].float().cpu().numpy()) <= 1e-2
-    assert rel_l2(a[2].cpu().numpy(), b[2].cpu().numpy()) <= 1e-2
+    b = res["simt"]
+    for path in ("tensor", "tensor_1cta"):
+        a = res[path]
+        assert (a[0].logp - b[0].logp).abs().max() <= 1e-4
+        assert (a[0].entropy - b[0].entropy).abs().max() <= 1e-4
+        assert rel_l2(a[1].float().cpu().numpy(), b[1].float().cpu().numpy()) <= 1e-2
+        assert rel_l2(a[2].cpu().numpy(), b[2].cpu().numpy()) <= 1e-2
+    # the two tensor-core variants differ only in how the vocabulary is split and merged
+    assert (res["tensor"][0].logp - res["tensor_1cta"][0].logp).abs().max() <= 1e-5
+    assert rel_l2(res["tensor"][1].float().cpu().numpy(), res["tensor_1cta"][1].float().cpu().numpy()) <= 1e-3
 
 
 # --------------------------------------------------------------------------- decision stage, bit exact
@@ -349,16 +368,16 @@ def test_repeated_runs_are_bit_identical():
 
 
 # --------------------------------------------------------------------------- active-row compaction
-@pytest.mark.parametrize("panel", [0, 256])
-def test_compacted_backward_matches_dense_and_oracle(panel):
+@pytest.mark.parametrize("panel,path", [(0, "auto"), (256, "auto"), (256, "tensor_1cta")])
+def test_compacted_backward_matches_dense_and_oracle(panel, path):
     """Rows with a zero coefficient (masked, clipped, zero advantage) are dropped from the backward
     contractions; the gradients must not change."""
     wl = synth.WORKLOADS["small"].scaled(T=1500, S=6, H=256, V=3000, lengths="lognormal:200:500", segment_len=64,
                                          planted=0.5, beta_planted=(100.0, 220.0), mpt_mode="always",
                                          noise="const:0.15", adv="bern:0.5:3")
     batch = synth.make_batch(wl, seed=33)
-    gp_d, op = both_params(batch, bwd_panel_tokens=panel)
-    gp_c, _ = both_params(batch, bwd_panel_tokens=panel, compact_rows=True)
+    gp_d, op = both_params(batch, bwd_panel_tokens=panel, kernel_path=path)
+    gp_c, _ = both_params(batch, bwd_panel_tokens=panel, compact_rows=True, kernel_path=path)
     out_d, dH_d, dW_d = gpu_fwd_bwd(batch, gp_d)
     out_c, dH_c, dW_c = gpu_fwd_bwd(batch, gp_c)
     st = out_c.stats_host()
@@ -426,10 +445,11 @@ def test_host_buffer_step_matches_device_calls(V, panel, compact):
                                pin(batch.seq_offsets), **ho)
 
 
-def test_kernel_timing_counts_the_tensor_core_launches():
+@pytest.mark.parametrize("path", ["tensor", "tensor_1cta"])
+def test_kernel_timing_counts_the_tensor_core_launches(path):
     wl = synth.WORKLOADS["small"].scaled(T=700, S=2, H=256, V=2048, lengths="tiny")
     batch = synth.make_batch(wl, seed=43)
-    gp, _ = both_params(batch, bwd_panel_tokens=256)
+    gp, _ = both_params(batch, bwd_panel_tokens=256, kernel_path=path)
     n0 = B.launch_count()
     B.kernel_timing_begin()
     gpu_fwd_bwd(batch, gp)
@@ -442,8 +462,7 @@ def test_kernel_timing_counts_the_tensor_core_launches():
 
 def B_panel_rows(gp):
     # panels are whole row tiles of the kernels in use (256 tokens for CTA pairs, 128 otherwise)
-    import os
-    unit = 128 if os.environ.get("ULORL_CTA_GROUP", "2").startswith("1") else 256
+    unit = 128 if gp.kernel_path == "tensor_1cta" else 256
     return -(-gp.bwd_panel_tokens // unit) * unit
 
 
