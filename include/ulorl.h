@@ -30,7 +30,8 @@
  *    inside the workspace and read back by ulorl_check_status(); offending rows are
  *    clamped, never read out of bounds.
  *  - Tokens are response tokens only; there is no ignore-index.
- *  - hidden, W and d_hidden have the element type `dtype`.  H must be a multiple of 8.
+ *  - hidden, W and d_hidden have the element type `dtype`.  H must be a multiple of 8, and
+ *    T ln(V + 1) < 2^29 (the range of the exact per-sequence entropy sums).
  */
 #ifndef ULORL_H_
 #define ULORL_H_
@@ -99,6 +100,9 @@ typedef struct {
                                /* to ulorl_workspace_bytes and to both calls.                                    */
   int32_t loss_norm;           /* ulorl_loss_norm_t: weight of a token's term in the loss                        */
   int32_t norm_seqs;           /* G of Eq. 5 for ULORL_NORM_SEQUENCE; 0 means num_seqs                           */
+  int32_t dw_dtype;            /* ulorl_dtype_t of d_W: F32 (default), or BF16 -- the sum over tokens is then    */
+                               /* still taken in float32 (in the workspace, which grows by 4 V H bytes) and      */
+                               /* rounded once when a row of d_W is final.  Part of the workspace size.          */
 } ulorl_params_t;
 
 typedef struct {
@@ -185,6 +189,29 @@ int ulorl_token_loss_decide_static(const ulorl_params_t* params,
                                    void* stats, void* cuda_stream);
 
 /*
+ * The mean entropy H-bar_i of Eq. 10 when a sequence is cut over several calls or ranks (token-range
+ * sharding of an ultra-long response).  The library keeps every per-sequence entropy sum as an exact
+ * 64-bit integer in units of 2^-34 nats, so pieces add up to the unsplit sum bit for bit:
+ *
+ *   ulorl_sequence_entropy_partials  from entropy[T] (the forward's output) and the call's seq_offsets,
+ *       fills table[total_seqs][2] = (entropy sum, token count) for the call's pieces -- piece k is global
+ *       sequence seq_ids[k] (NULL: k) -- and zeros elsewhere.  Tables of all calls / ranks are then added
+ *       element by element (an int64 SUM all-reduce).
+ *   ulorl_sequence_entropy_combine   from the summed table, writes seq_entropy[k] = mean of sequence
+ *       seq_ids[k], k < num_seqs, in float32 with the arithmetic of the forward call (the value an unsplit
+ *       call returns), and optionally batch_entropy[0] = token mean over all sequences.  These go to
+ *       ulorl_token_loss_decide as entropy_supplied (ent_scope = SUPPLIED).
+ *
+ * All pointers are device memory.  workspace may be NULL; if given, its status word reports offsets or
+ * ids out of range (they are skipped).
+ */
+int ulorl_sequence_entropy_partials(const ulorl_params_t* params, const float* entropy,
+                                    const int32_t* seq_offsets, const int32_t* seq_ids, int32_t total_seqs,
+                                    int64_t* table, void* workspace, void* cuda_stream);
+int ulorl_sequence_entropy_combine(const int64_t* table, int32_t total_seqs, const int32_t* seq_ids,
+                                   int32_t num_seqs, float* seq_entropy, float* batch_entropy, void* cuda_stream);
+
+/*
  * Group-normalised advantages (Eq. 4) for responses stored group after group (`group_size` responses
  * per prompt, the last group may be shorter): advantages[i] = (R_i - mean) / std over the group,
  * population standard deviation, 0 for a group without spread.  keep[i] (optional) is 1 when the
@@ -197,16 +224,38 @@ int ulorl_group_advantages(const float* rewards, int32_t num_responses, int32_t 
 
 /*
  * Backward (chain rule through Eq. 6): with dz[t,v] = kappa * grad_loss * grad_coef[t] *
- * (1[v = y_t] - exp(z[t,v] - lse[t])), writes d_hidden[T,H] (params->dtype) and d_W[V,H] (f32;
- * added into when params->dw_accumulate).  grad_loss is a device scalar or NULL (= 1).
- * Logits are recomputed tile by tile; nothing of size T x V is kept beyond one token panel
- * of dz in the workspace.
+ * (1[v = y_t] - exp(z[t,v] - lse[t])), writes d_hidden[T,H] (params->dtype) and d_W[V,H]
+ * (params->dw_dtype, f32 by default; added into when params->dw_accumulate).  grad_loss is a
+ * device scalar or NULL (= 1).  Logits are recomputed tile by tile; nothing of size T x V is kept
+ * beyond one token panel of dz in the workspace.
  */
 int ulorl_token_loss_bwd(const ulorl_params_t* params,
                          const void* hidden, const void* W, const int32_t* targets,
                          const float* lse, const float* grad_coef, const float* grad_loss,
-                         void* d_hidden, float* d_W,
+                         void* d_hidden, void* d_W,
                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * The same backward for a caller that wants to start moving d_W before the pass is over -- the sum of
+ * d_W over data-parallel ranks (the one exchange of the update of Algorithm 1 when whole sequences are
+ * sharded), or a copy to the host.  d_W is a sum over all tokens, so its rows are final only while the
+ * LAST token panel is processed; there the library computes d_W before d_hidden and in slabs of
+ * vocabulary rows (whole waves of tiles, about eight slabs), and calls
+ *     on_slab(user, first_row, rows)
+ * on the calling host thread right after the launches that make rows [first_row, first_row + rows)
+ * of d_W final have been put on cuda_stream.  Nothing has run yet at that point: the callback orders
+ * its own work behind those launches (record an event on cuda_stream and make another stream wait for
+ * it, or start a collective that orders itself after cuda_stream) and returns; the d_hidden launches of
+ * the panel follow on cuda_stream and overlap with it.  The slabs come in ascending row order and cover
+ * [0, V) once.  A non-zero return value stops the pass and is returned.  on_slab = NULL gives
+ * ulorl_token_loss_bwd.  Results are those of ulorl_token_loss_bwd bit for bit.
+ */
+typedef int (*ulorl_dw_slab_fn)(void* user, int32_t first_row, int32_t rows);
+int ulorl_token_loss_bwd_slabs(const ulorl_params_t* params,
+                               const void* hidden, const void* W, const int32_t* targets,
+                               const float* lse, const float* grad_coef, const float* grad_loss,
+                               void* d_hidden, void* d_W, ulorl_dw_slab_fn on_slab, void* user,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* Synchronises the stream, reads the workspace status word and returns it: ULORL_OK, or
  * ULORL_ERR_DEVICE_TIMEOUT, ULORL_ERR_INVALID_ARG (seq_offsets on the device were not
@@ -233,7 +282,7 @@ int ulorl_kernel_timing_end(float* total_ms, int64_t* launches);
  * HOST memory (pinned memory makes the copies asynchronous).  Inputs h_* are copied to the device
  * arena, both passes run there, and every non-NULL output is copied back: h_logp[T], h_entropy[T],
  * h_flags[T], h_seq_entropy[S], h_loss[1], h_stats (ulorl_stats_t), h_d_hidden[T,H] (params->dtype),
- * h_d_W[V,H] (f32).  d_arena is DEVICE memory of at least ulorl_host_step_arena_bytes(params)
+ * h_d_W[V,H] (params->dw_dtype).  d_arena is DEVICE memory of at least ulorl_host_step_arena_bytes(params)
  * bytes, owned by the caller and reusable across calls; it holds the device copies, the outputs
  * and the workspace.  Asynchronous on cuda_stream: synchronise the stream before reading outputs
  * or reusing the host buffers.  Copies are overlapped with the passes: hidden states arrive in
@@ -251,7 +300,7 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params,
                                const float* h_advantages, const int32_t* h_seq_offsets,
                                const float* h_entropy_supplied,
                                float* h_logp, float* h_entropy, uint8_t* h_flags, float* h_seq_entropy,
-                               float* h_loss, void* h_stats, void* h_d_hidden, float* h_d_W,
+                               float* h_loss, void* h_stats, void* h_d_hidden, void* h_d_W,
                                void* d_arena, size_t arena_bytes, void* cuda_stream);
 
 #ifdef __cplusplus

@@ -46,6 +46,7 @@ class CParams(ctypes.Structure):
         ("norm_tokens", ctypes.c_int64), ("current_version", ctypes.c_int32),
         ("dw_accumulate", ctypes.c_int32), ("kernel_path", ctypes.c_int32), ("bwd_panel_tokens", ctypes.c_int32),
         ("compact_rows", ctypes.c_int32), ("loss_norm", ctypes.c_int32), ("norm_seqs", ctypes.c_int32),
+        ("dw_dtype", ctypes.c_int32),
     ]
 
 
@@ -61,11 +62,15 @@ class CStats(ctypes.Structure):
 
 
 EXPORTS = ("ulorl_workspace_bytes", "ulorl_token_loss_fwd", "ulorl_token_loss_decide", "ulorl_token_loss_bwd",
+           "ulorl_token_loss_bwd_slabs",
            "ulorl_check_status", "ulorl_status_string", "ulorl_launch_count", "ulorl_kernel_timing_begin",
            "ulorl_kernel_timing_end", "ulorl_host_step_arena_bytes", "ulorl_token_loss_step_host",
-           "ulorl_token_loss_decide_static", "ulorl_group_advantages")
+           "ulorl_token_loss_decide_static", "ulorl_group_advantages", "ulorl_sequence_entropy_partials",
+           "ulorl_sequence_entropy_combine")
 STATIC_MAX_TOKENS, STATIC_MAX_SEQS = 1 << 20, 1 << 16
 KERNEL_KINDS = ("stats", "dz", "d_hidden", "d_W")
+
+DW_SLAB_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32)
 
 _lib = None
 
@@ -90,8 +95,14 @@ def load_library() -> ctypes.CDLL:
     lib.ulorl_token_loss_decide_static.argtypes = [cp] + [vp] * 12 + [vp]
     lib.ulorl_group_advantages.restype = ctypes.c_int
     lib.ulorl_group_advantages.argtypes = [vp, ctypes.c_int32, ctypes.c_int32, vp, vp, vp]
+    lib.ulorl_sequence_entropy_partials.restype = ctypes.c_int
+    lib.ulorl_sequence_entropy_partials.argtypes = [cp, vp, vp, vp, ctypes.c_int32, vp, vp, vp]
+    lib.ulorl_sequence_entropy_combine.restype = ctypes.c_int
+    lib.ulorl_sequence_entropy_combine.argtypes = [vp, ctypes.c_int32, vp, ctypes.c_int32, vp, vp, vp]
     lib.ulorl_token_loss_bwd.restype = ctypes.c_int
     lib.ulorl_token_loss_bwd.argtypes = [cp] + [vp] * 8 + [vp, ctypes.c_size_t, vp]
+    lib.ulorl_token_loss_bwd_slabs.restype = ctypes.c_int
+    lib.ulorl_token_loss_bwd_slabs.argtypes = [cp] + [vp] * 8 + [DW_SLAB_FN, vp] + [vp, ctypes.c_size_t, vp]
     lib.ulorl_check_status.restype = ctypes.c_int
     lib.ulorl_check_status.argtypes = [vp, vp]
     lib.ulorl_status_string.restype = ctypes.c_char_p
@@ -144,6 +155,11 @@ class Params:
     compact_rows: bool = False
     loss_norm: str = "tokens"
     norm_seqs: int = 0
+    dw_dtype: str = "f32"
+
+    @property
+    def dw_torch_dtype(self):
+        return torch.bfloat16 if self.dw_dtype == "bf16" else torch.float32
 
     def to_c(self) -> CParams:
         return CParams(self.T, self.H, self.V, self.num_seqs, BF16 if self.dtype == "bf16" else F32,
@@ -151,7 +167,7 @@ class Params:
                        self.clip_eps_low, self.clip_eps_high, self.mpt_tau, self.entropy_target,
                        self.inv_temperature, self.norm_tokens, self.current_version, int(self.dw_accumulate),
                        _PATH[self.kernel_path], self.bwd_panel_tokens, int(self.compact_rows),
-                       _NORM[self.loss_norm], self.norm_seqs)
+                       _NORM[self.loss_norm], self.norm_seqs, BF16 if self.dw_dtype == "bf16" else F32)
 
 
 def workspace_bytes(p: Params) -> int:
@@ -283,20 +299,36 @@ def token_loss_decide_static(p: Params, logp, entropy, old_logp, segment_version
 
 
 def token_loss_bwd(p: Params, hidden, W, targets, lse, grad_coef, grad_loss=None, d_hidden=None, d_W=None,
-                   workspace: Optional[torch.Tensor] = None):
-    """ulorl_token_loss_bwd on the current CUDA stream.  Returns (d_hidden, d_W)."""
+                   workspace: Optional[torch.Tensor] = None, on_dw_slab=None):
+    """ulorl_token_loss_bwd on the current CUDA stream.  Returns (d_hidden, d_W).  With on_dw_slab (a callable
+    (first_row, rows) -> None) the call goes through ulorl_token_loss_bwd_slabs: the callable runs on this
+    thread each time the launches that make a slab of rows of d_W final have been queued."""
     lib = load_library()
     dev = hidden.device
     if d_hidden is None:
         d_hidden = torch.empty_like(hidden)
     if d_W is None:
-        d_W = torch.zeros(p.V, p.H, dtype=torch.float32, device=dev) if p.dw_accumulate else \
-            torch.empty(p.V, p.H, dtype=torch.float32, device=dev)
-    _want(d_W, torch.float32, p.V * p.H, "d_W")
+        d_W = (torch.zeros if p.dw_accumulate else torch.empty)(p.V, p.H, dtype=p.dw_torch_dtype, device=dev)
+    _want(d_W, p.dw_torch_dtype, p.V * p.H, "d_W")
     workspace = workspace if workspace is not None else alloc_workspace(p, dev)
-    code = lib.ulorl_token_loss_bwd(
-        ctypes.byref(p.to_c()), _ptr(hidden), _ptr(W), _ptr(targets), _ptr(lse), _ptr(grad_coef), _ptr(grad_loss),
-        _ptr(d_hidden), _ptr(d_W), _ptr(workspace), workspace.numel(), _stream())
+    head = (ctypes.byref(p.to_c()), _ptr(hidden), _ptr(W), _ptr(targets), _ptr(lse), _ptr(grad_coef), _ptr(grad_loss),
+            _ptr(d_hidden), _ptr(d_W))
+    tail = (_ptr(workspace), workspace.numel(), _stream())
+    if on_dw_slab is None:
+        code = lib.ulorl_token_loss_bwd(*head, *tail)
+    else:
+        failure = []
+
+        def trampoline(_user, first_row, rows):
+            try:
+                on_dw_slab(int(first_row), int(rows))
+                return 0
+            except BaseException as exc:       # an exception cannot cross the C frames: stop the pass, re-raise below
+                failure.append(exc)
+                return -4
+        code = lib.ulorl_token_loss_bwd_slabs(*head, DW_SLAB_FN(trampoline), None, *tail)
+        if failure:
+            raise failure[0]
     _check(code, "ulorl_token_loss_bwd")
     return d_hidden, d_W
 
@@ -343,6 +375,36 @@ def token_loss_step_host(p: Params, arena: torch.Tensor, hidden, W, targets, old
         _hptr(seq_entropy), _hptr(loss), _hptr(stats), _hptr(d_hidden), _hptr(d_W), _ptr(arena), arena.numel(),
         _stream())
     _check(code, "ulorl_token_loss_step_host")
+
+
+def sequence_entropy_partials(p: Params, entropy: torch.Tensor, seq_offsets: torch.Tensor, seq_ids, total_seqs: int,
+                              workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """ulorl_sequence_entropy_partials: int64 [total_seqs, 2] (entropy sum in 2^-34 nats, token count) of the
+    call's pieces of sequences, zero for the sequences it holds nothing of."""
+    _want(entropy, torch.float32, p.T, "entropy")
+    _want(seq_offsets, torch.int32, p.num_seqs + 1, "seq_offsets")
+    if seq_ids is not None:
+        _want(seq_ids, torch.int32, p.num_seqs, "seq_ids")
+    table = torch.empty(total_seqs, 2, dtype=torch.int64, device=entropy.device)
+    code = load_library().ulorl_sequence_entropy_partials(ctypes.byref(p.to_c()), _ptr(entropy), _ptr(seq_offsets),
+                                                          _ptr(seq_ids), total_seqs, _ptr(table), _ptr(workspace),
+                                                          _stream())
+    _check(code, "ulorl_sequence_entropy_partials")
+    return table
+
+
+def sequence_entropy_combine(table: torch.Tensor, seq_ids, num_seqs: int, want_batch: bool = False):
+    """ulorl_sequence_entropy_combine: float32 mean entropy of the sequences seq_ids (None: the first num_seqs)
+    from a summed table; with want_batch also the token mean over the whole table."""
+    _want(table, torch.int64, table.numel(), "table")
+    if seq_ids is not None:
+        _want(seq_ids, torch.int32, num_seqs, "seq_ids")
+    out = torch.empty(max(num_seqs, 1), dtype=torch.float32, device=table.device)
+    batch = torch.empty(1, dtype=torch.float32, device=table.device) if want_batch else None
+    code = load_library().ulorl_sequence_entropy_combine(_ptr(table), table.shape[0], _ptr(seq_ids), num_seqs,
+                                                         _ptr(out), _ptr(batch), _stream())
+    _check(code, "ulorl_sequence_entropy_combine")
+    return (out[:num_seqs], batch) if want_batch else out[:num_seqs]
 
 
 def group_advantages(rewards: torch.Tensor, group_size: int):

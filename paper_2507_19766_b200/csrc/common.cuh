@@ -35,6 +35,17 @@ struct DecideConsts {
   int is_mode, mpt_mode, ent_scope, adv_per_token, current_version, loss_norm;
 };
 
+// Per-sequence entropy sums (H-bar of Eq. 10) are kept as 64-bit integers in units of 2^-kEntropyFixShift
+// nats: integer addition is associative, so the sum of a sequence does not depend on the order of its
+// tokens, on how a launch spreads them over threads, or on how a token-range sharding cuts the
+// sequence over ranks -- an integer all-reduce of the pieces gives the unsplit sum bit for bit.  One
+// token is rounded by at most 2^-35 nats (its float32 entropy carries 2^-24 relative), and a sum holds
+// up to 2^29 nats, which the host checks against T ln V.
+constexpr int kEntropyFixShift = 34;
+constexpr double kEntropyFixScale = 17179869184.0;          // 2^34
+constexpr double kEntropyFixInv = 1.0 / 17179869184.0;
+constexpr double kEntropyFixCapacity = 536870912.0;         // 2^29 nats per sum (2^63 / 2^34)
+
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 }  // namespace ulorl

@@ -36,43 +36,104 @@ __global__ void merge_splits_kernel(int T, int n_split, float kappa, const float
 }
 
 // ------------------------------------------------------------------------------------------
-// H-bar_i of Eq. 10: mean per-token entropy of each sequence.  One block per sequence, float64
-// accumulation in a fixed order (thread-strided partial sums, then a fixed tree).
+// H-bar_i of Eq. 10: mean per-token entropy of each sequence.  One block per sequence; the sum is
+// an exact 64-bit integer sum of the entropies in units of 2^-34 nats (common.cuh), so it is the
+// same whatever the order, and a sequence cut over several calls or ranks adds up to the same bits.
 // ------------------------------------------------------------------------------------------
 constexpr int kSeqThreads = 256;
 
-__global__ void seq_entropy_kernel(int S, int T, const int* __restrict__ seq_offsets, const float* __restrict__ entropy,
-                                   double* __restrict__ seq_sum, float* __restrict__ seq_entropy, int* __restrict__ status) {
-  __shared__ double red[kSeqThreads];
-  const int i = blockIdx.x;
-  int a = seq_offsets[i], b = seq_offsets[i + 1];
-  // offsets are device data the host never saw: a bad pair is reported and clamped, never followed out of range
-  const bool bad = a < 0 || b < a || b > T || (i == 0 && a != 0) || (i == S - 1 && b != T);
-  if (bad) {
-    if (threadIdx.x == 0) atomicOr(status, kStatusBadOffsets);
-    a = a < 0 ? 0 : (a > T ? T : a);
-    b = b < a ? a : (b > T ? T : b);
-  }
-  double acc = 0.0;
-  for (int t = a + threadIdx.x; t < b; t += kSeqThreads) acc += (double)entropy[t];
+__device__ __forceinline__ long long entropy_to_fixed(float e) {
+  // NaN counts as 0 and absurd magnitudes are clipped, so that the conversion is always defined
+  const float c = (e == e) ? fminf(fmaxf(e, -1024.f), 1024.f) : 0.f;
+  return __double2ll_rn((double)c * kEntropyFixScale);
+}
+__device__ __forceinline__ float fixed_mean(long long sum, long long count) {
+  return count > 0 ? (float)(((double)sum * kEntropyFixInv) / (double)count) : 0.f;
+}
+
+// Sum over tokens [a, b) of one sequence by the whole block; the result is valid in thread 0.
+__device__ __forceinline__ long long block_entropy_sum(const float* __restrict__ entropy, int a, int b) {
+  __shared__ long long red[kSeqThreads];
+  long long acc = 0;
+  for (int t = a + threadIdx.x; t < b; t += kSeqThreads) acc += entropy_to_fixed(entropy[t]);
   red[threadIdx.x] = acc;
   __syncthreads();
   for (int w = kSeqThreads / 2; w > 0; w >>= 1) {
     if (threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
     __syncthreads();
   }
-  if (threadIdx.x == 0) {
-    seq_sum[i] = red[0];
-    if (seq_entropy) seq_entropy[i] = b > a ? (float)(red[0] / (double)(b - a)) : 0.f;
+  return red[0];
+}
+
+// Offsets are device data the host never saw: a bad pair is reported and clamped, never followed out of range.
+__device__ __forceinline__ void checked_range(const int* __restrict__ seq_offsets, int i, int S, int T, int& a, int& b,
+                                              int* __restrict__ status) {
+  a = seq_offsets[i];
+  b = seq_offsets[i + 1];
+  const bool bad = a < 0 || b < a || b > T || (i == 0 && a != 0) || (i == S - 1 && b != T);
+  if (bad) {
+    if (threadIdx.x == 0 && status) atomicOr(status, kStatusBadOffsets);
+    a = a < 0 ? 0 : (a > T ? T : a);
+    b = b < a ? a : (b > T ? T : b);
   }
 }
 
-// Token mean of the entropy over the whole call: the sequence sums added in sequence order.
-__global__ void batch_entropy_kernel(int S, int T, const double* __restrict__ seq_sum, float* __restrict__ batch_mean) {
+__global__ void seq_entropy_kernel(int S, int T, const int* __restrict__ seq_offsets, const float* __restrict__ entropy,
+                                   long long* __restrict__ seq_sum, float* __restrict__ seq_entropy, int* __restrict__ status) {
+  const int i = blockIdx.x;
+  int a, b;
+  checked_range(seq_offsets, i, S, T, a, b, status);
+  const long long sum = block_entropy_sum(entropy, a, b);
+  if (threadIdx.x == 0) {
+    seq_sum[i] = sum;
+    if (seq_entropy) seq_entropy[i] = fixed_mean(sum, (long long)(b - a));
+  }
+}
+
+// Token mean of the entropy over the whole call: the (exact) sum of the sequence sums.
+__global__ void batch_entropy_kernel(int S, int T, const long long* __restrict__ seq_sum, float* __restrict__ batch_mean) {
   if (threadIdx.x == 0 && blockIdx.x == 0) {
-    double tot = 0.0;
+    long long tot = 0;
     for (int i = 0; i < S; ++i) tot += seq_sum[i];
-    *batch_mean = T > 0 ? (float)(tot / (double)T) : 0.f;
+    *batch_mean = fixed_mean(tot, (long long)T);
+  }
+}
+
+// The pieces of sequences that one call holds, as rows (sum, count) of a table over ALL sequences of the
+// step: piece k of the call is sequence seq_ids[k] (k itself without seq_ids).  Rows of other sequences
+// stay as the caller's memset left them; tables of several calls or ranks add up element by element.
+__global__ void seq_entropy_partials_kernel(int S, int T, const int* __restrict__ seq_offsets,
+                                            const float* __restrict__ entropy, const int* __restrict__ seq_ids,
+                                            int total_seqs, long long* __restrict__ table, int* __restrict__ status) {
+  const int k = blockIdx.x;
+  int a, b;
+  checked_range(seq_offsets, k, S, T, a, b, status);
+  const long long sum = block_entropy_sum(entropy, a, b);
+  if (threadIdx.x == 0) {
+    const int id = seq_ids ? seq_ids[k] : k;
+    if (id < 0 || id >= total_seqs) {
+      if (status) atomicOr(status, kStatusBadOffsets);
+    } else {                                   // pieces of one sequence inside one call are added, too
+      atomicAdd(reinterpret_cast<unsigned long long*>(table + 2 * (size_t)id), (unsigned long long)sum);
+      atomicAdd(reinterpret_cast<unsigned long long*>(table + 2 * (size_t)id + 1), (unsigned long long)(b - a));
+    }
+  }
+}
+
+// Means of the sequences seq_ids[0..n) from a summed table, with the arithmetic of seq_entropy_kernel:
+// a sequence whose pieces were summed here gets the float32 mean the unsplit call would have given it.
+__global__ void seq_entropy_combine_kernel(int n, const int* __restrict__ seq_ids, int total_seqs,
+                                           const long long* __restrict__ table, float* __restrict__ seq_entropy,
+                                           float* __restrict__ batch_entropy) {
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k < n) {
+    const int id = seq_ids ? seq_ids[k] : k;
+    seq_entropy[k] = (id >= 0 && id < total_seqs) ? fixed_mean(table[2 * (size_t)id], table[2 * (size_t)id + 1]) : 0.f;
+  }
+  if (batch_entropy && k == 0) {
+    long long tot = 0, cnt = 0;
+    for (int i = 0; i < total_seqs; ++i) { tot += table[2 * (size_t)i]; cnt += table[2 * (size_t)i + 1]; }
+    *batch_entropy = fixed_mean(tot, cnt);
   }
 }
 
@@ -291,6 +352,35 @@ __global__ void group_advantage_kernel(int S, int group, const float* __restrict
   for (int i = a; i < b; ++i) {
     adv[i] = sd > 0.0 ? (float)(((double)rewards[i] - mean) / sd) : 0.f;
     if (keep) keep[i] = kept;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// bf16 d_W: rows of the float32 sum over tokens that are final are rounded once (round to nearest
+// even) into the caller's array, eight elements a thread; with `accumulate` the caller's values are
+// added first.
+// ------------------------------------------------------------------------------------------
+__global__ void dw_round_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ out, size_t n8, int accumulate) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += (size_t)gridDim.x * blockDim.x) {
+    const float4 a0 = reinterpret_cast<const float4*>(acc)[2 * i];
+    const float4 a1 = reinterpret_cast<const float4*>(acc)[2 * i + 1];
+    float v[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+    uint4* dst = reinterpret_cast<uint4*>(out) + i;
+    if (accumulate) {
+      const uint4 old = *dst;
+      const __nv_bfloat162* o = reinterpret_cast<const __nv_bfloat162*>(&old);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float2 f = __bfloat1622float2(o[j]);
+        v[2 * j] += f.x;
+        v[2 * j + 1] += f.y;
+      }
+    }
+    uint4 r;
+    __nv_bfloat162* rp = reinterpret_cast<__nv_bfloat162*>(&r);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) rp[j] = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+    *dst = r;
   }
 }
 

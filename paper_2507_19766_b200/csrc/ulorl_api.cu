@@ -67,6 +67,8 @@ struct Plan {
   size_t t_pad;           // rows of the compacted buffers
   size_t off_n_active, off_blk_count, off_blk_offset, off_position, off_targets_c, off_lse_c, off_coef_c,
       off_hidden_c, off_dh_c;
+  bool dw_bf16;           // d_W leaves as bf16: the float32 sum over tokens is kept at off_dw_acc
+  size_t off_dw_acc;
   int decide_blocks;
 };
 
@@ -93,7 +95,10 @@ static int validate_params(const ulorl_params_t* p) {
   if (!(p->mpt_tau > 0.f) || p->mpt_tau > 1.f) return ULORL_ERR_INVALID_ARG;
   if (p->norm_tokens < 0 || p->bwd_panel_tokens < 0) return ULORL_ERR_INVALID_ARG;
   if (p->compact_rows != 0 && p->compact_rows != 1) return ULORL_ERR_INVALID_ARG;
+  if (p->dw_dtype != ULORL_F32 && p->dw_dtype != ULORL_BF16) return ULORL_ERR_INVALID_ARG;
   if (p->H % 8 != 0) return ULORL_ERR_UNSUPPORTED;
+  // the exact integer entropy sums hold 2^29 nats; no token's entropy exceeds ln V
+  if ((double)p->T * std::log((double)p->V + 1.0) >= kEntropyFixCapacity) return ULORL_ERR_UNSUPPORTED;
   return ULORL_OK;
 }
 
@@ -151,7 +156,7 @@ static Plan make_plan(const ulorl_params_t* p) {
   size_t off = 0;
   pl.off_status = off;      off += 256;
   pl.off_batch_mean = pl.off_status + 16;
-  pl.off_seq_sum = off;     off = align_up(off + sizeof(double) * (size_t)(p->num_seqs > 0 ? p->num_seqs : 1), 256);
+  pl.off_seq_sum = off;     off = align_up(off + sizeof(long long) * (size_t)(p->num_seqs > 0 ? p->num_seqs : 1), 256);
   pl.off_partials = off;    off = align_up(off + sizeof(float4) * (size_t)pl.n_split * (size_t)(T > 0 ? T : 1), 256);
   pl.off_acc_y = off;       off = align_up(off + sizeof(float) * (size_t)(T > 0 ? T : 1), 256);
   pl.off_decide = off;      off = align_up(off + sizeof(DecidePartial) * (size_t)(pl.decide_blocks > 0 ? pl.decide_blocks : 1), 1024);
@@ -170,6 +175,11 @@ static Plan make_plan(const ulorl_params_t* p) {
     pl.off_coef_c = off;     off = align_up(off + 4 * pl.t_pad, 256);
     pl.off_hidden_c = off;   off = align_up(off + 2 * pl.t_pad * (size_t)p->H, 1024);
     pl.off_dh_c = off;       off = align_up(off + 2 * pl.t_pad * (size_t)p->H, 1024);
+  }
+  pl.dw_bf16 = p->dw_dtype == ULORL_BF16;
+  if (pl.dw_bf16) {
+    pl.off_dw_acc = off;
+    off = align_up(off + sizeof(float) * (size_t)V * (size_t)p->H, 1024);
   }
   pl.total = off;
   return pl;
@@ -356,7 +366,7 @@ static int run_decide(const ulorl_params_t* p, const Plan& pl, const float* logp
   const int T = p->T, S = p->num_seqs;
   int* status = reinterpret_cast<int*>(ws + pl.off_status);
   float* batch_mean = reinterpret_cast<float*>(ws + pl.off_batch_mean);
-  double* seq_sum = reinterpret_cast<double*>(ws + pl.off_seq_sum);
+  long long* seq_sum = reinterpret_cast<long long*>(ws + pl.off_seq_sum);
   DecidePartial* partials = reinterpret_cast<DecidePartial*>(ws + pl.off_decide);
   // the gate needs a float array of per-sequence means even when the caller does not want it back
   float* seq_ent_out = seq_entropy;
@@ -554,27 +564,50 @@ int ulorl_token_loss_fwd(const ulorl_params_t* params, const void* hidden, const
                   nullptr);
 }
 
+// d_W rows [v0, v0 + v_rows) are final in the float32 accumulator: round them into the caller's bf16 d_W.
+static int round_dw_rows(const float* acc, void* d_W, int v0, int v_rows, int H, int accumulate, cudaStream_t stream) {
+  const size_t n8 = (size_t)v_rows * (size_t)H / 8;            // H is a multiple of 8
+  if (n8 == 0) return ULORL_OK;
+  const size_t first = (size_t)v0 * (size_t)H;
+  const unsigned blocks = (unsigned)std::min<size_t>((n8 + 255) / 256, 148u * 16u);
+  dw_round_kernel<<<blocks, 256, 0, stream>>>(acc + first, static_cast<__nv_bfloat16*>(d_W) + first, n8, accumulate);
+  return check_launch();
+}
+
 static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void* W, const int32_t* targets,
-                    const float* lse, const float* grad_coef, const float* grad_loss, void* d_hidden, float* d_W,
+                    const float* lse, const float* grad_coef, const float* grad_loss, void* d_hidden, void* d_W_out,
                     void* workspace, size_t workspace_bytes, void* cuda_stream, const StepHooks* hooks) {
   int st = validate_params(params);
   if (st != ULORL_OK) return st;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   const int T = params->T, H = params->H, V = params->V;
+  const size_t dw_elem = params->dw_dtype == ULORL_BF16 ? 2 : 4;
   if (T == 0) {
-    if (!d_W) return ULORL_ERR_INVALID_ARG;
-    if (!params->dw_accumulate && cudaMemsetAsync(d_W, 0, sizeof(float) * (size_t)V * H, stream) != cudaSuccess)
+    if (!d_W_out) return ULORL_ERR_INVALID_ARG;
+    if (!params->dw_accumulate && cudaMemsetAsync(d_W_out, 0, dw_elem * (size_t)V * H, stream) != cudaSuccess)
       return ULORL_ERR_CUDA;
+    if (hooks && hooks->after_dw_slab) return hooks->after_dw_slab(0, V);
     return ULORL_OK;
   }
-  if (!hidden || !W || !targets || !lse || !grad_coef || !d_hidden || !d_W || !workspace) return ULORL_ERR_INVALID_ARG;
-  if (!aligned16(hidden) || !aligned16(W) || !aligned16(d_hidden) || !aligned16(d_W) || !aligned16(workspace))
+  if (!hidden || !W || !targets || !lse || !grad_coef || !d_hidden || !d_W_out || !workspace) return ULORL_ERR_INVALID_ARG;
+  if (!aligned16(hidden) || !aligned16(W) || !aligned16(d_hidden) || !aligned16(d_W_out) || !aligned16(workspace))
     return ULORL_ERR_UNSUPPORTED;
   const Plan pl = make_plan(params);
   if (workspace_bytes < pl.total) return ULORL_ERR_WORKSPACE;
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
   const float kappa = params->inv_temperature;
   int* status = reinterpret_cast<int*>(ws + pl.off_status);
+  // The contractions sum d_W in float32: straight into the caller's array, or, for a bf16 d_W, into the
+  // workspace, from where rows are rounded (and added to the caller's values, if asked) once they are final.
+  float* d_W = pl.dw_bf16 ? reinterpret_cast<float*>(ws + pl.off_dw_acc) : static_cast<float*>(d_W_out);
+  const int acc_into = pl.dw_bf16 ? 0 : params->dw_accumulate;
+  auto dw_rows_final = [&](int v0, int v_rows) -> int {
+    if (pl.dw_bf16) {
+      const int rc = round_dw_rows(d_W, d_W_out, v0, v_rows, H, params->dw_accumulate, stream);
+      if (rc != ULORL_OK) return rc;
+    }
+    return (hooks && hooks->after_dw_slab) ? hooks->after_dw_slab(v0, v_rows) : (int)ULORL_OK;
+  };
 
   if (pl.tensor) {
     __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(ws + pl.off_dz);
@@ -601,7 +634,7 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
           T, H, grad_coef, blk_offset, n_act, static_cast<const __nv_bfloat16*>(hidden), targets, lse, position,
           hidden_c, targets_c, lse_c, coef_c);
       ULORL_LAUNCH_CHECK();
-      if (!params->dw_accumulate && cudaMemsetAsync(d_W, 0, sizeof(float) * (size_t)V * H, stream) != cudaSuccess)
+      if (!acc_into && cudaMemsetAsync(d_W, 0, sizeof(float) * (size_t)V * H, stream) != cudaSuccess)
         return ULORL_ERR_CUDA;
       n_active = n_act;
       hidden = hidden_c;
@@ -679,7 +712,7 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
         a.row0 = v0;
         a.d_W = d_W;
         a.out_ld = (size_t)H;
-        a.accumulate = (panel > 0 || params->dw_accumulate || pl.compact) ? 1 : 0;
+        a.accumulate = (panel > 0 || acc_into || pl.compact) ? 1 : 0;
         a.dyn_rows = n_active; a.dyn_base = t0;
         a.status = status;
         return launch_umma<kModeDW>(pl, map_dz_mn, map_hidden_mn, map_dw_out, a, stream);
@@ -696,7 +729,7 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
           const int v_rows = (V - v0) < slab_rows ? (V - v0) : slab_rows;
           st = run_d_W(v0, v_rows);
           if (st != ULORL_OK) return st;
-          st = hooks->after_dw_slab(v0, v_rows);
+          st = dw_rows_final(v0, v_rows);
           if (st != ULORL_OK) return st;
         }
         st = run_d_hidden();
@@ -706,6 +739,10 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
         if (st != ULORL_OK) return st;
         st = run_d_W(0, V);
         if (st != ULORL_OK) return st;
+        if (last_panel) {
+          st = dw_rows_final(0, V);
+          if (st != ULORL_OK) return st;
+        }
       }
     }
     if (pl.compact) {
@@ -724,7 +761,7 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
     const dim3 gdz((rows + kSimtTile - 1) / kSimtTile, (V + kSimtTile - 1) / kSimtTile);
     const dim3 gdh((H + kSimtTile - 1) / kSimtTile, (rows + kSimtTile - 1) / kSimtTile);
     const dim3 gdw((H + kSimtTile - 1) / kSimtTile, (V + kSimtTile - 1) / kSimtTile);
-    const int acc = (panel > 0 || params->dw_accumulate) ? 1 : 0;
+    const int acc = (panel > 0 || acc_into) ? 1 : 0;
     if (params->dtype == ULORL_F32) {
       const float* h = static_cast<const float*>(hidden);
       const float* w = static_cast<const float*>(W);
@@ -756,23 +793,36 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
       if (st != ULORL_OK) return st;
     }
   }
-  return ULORL_OK;
+  return dw_rows_final(0, V);
 }
 
 int ulorl_token_loss_bwd(const ulorl_params_t* params, const void* hidden, const void* W, const int32_t* targets,
-                         const float* lse, const float* grad_coef, const float* grad_loss, void* d_hidden, float* d_W,
+                         const float* lse, const float* grad_coef, const float* grad_loss, void* d_hidden, void* d_W,
                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
   return bwd_impl(params, hidden, W, targets, lse, grad_coef, grad_loss, d_hidden, d_W, workspace, workspace_bytes,
                   cuda_stream, nullptr);
+}
+
+int ulorl_token_loss_bwd_slabs(const ulorl_params_t* params, const void* hidden, const void* W, const int32_t* targets,
+                               const float* lse, const float* grad_coef, const float* grad_loss, void* d_hidden,
+                               void* d_W, ulorl_dw_slab_fn on_slab, void* user, void* workspace,
+                               size_t workspace_bytes, void* cuda_stream) {
+  if (!on_slab)
+    return bwd_impl(params, hidden, W, targets, lse, grad_coef, grad_loss, d_hidden, d_W, workspace, workspace_bytes,
+                    cuda_stream, nullptr);
+  StepHooks hooks;
+  hooks.after_dw_slab = [&](int v0, int v_rows) { return on_slab(user, (int32_t)v0, (int32_t)v_rows); };
+  return bwd_impl(params, hidden, W, targets, lse, grad_coef, grad_loss, d_hidden, d_W, workspace, workspace_bytes,
+                  cuda_stream, &hooks);
 }
 
 // ------------------------------------------------------------------ decision stage without a workspace
 // Scratch of ulorl_token_loss_decide_static: a fixed array in the library's own device image,
 // resident on every GPU that loads the library until the process exits.
 //   [0, 256)                       status word and batch-mean slot
-//   [256, 256 + 8 * max seqs)      float64 entropy sum per sequence
+//   [256, 256 + 8 * max seqs)      64-bit integer entropy sum per sequence
 //   rest                           one DecidePartial per block of 256 tokens
-constexpr size_t kStaticSeqBytes = sizeof(double) * (size_t)ULORL_STATIC_MAX_SEQS;
+constexpr size_t kStaticSeqBytes = sizeof(long long) * (size_t)ULORL_STATIC_MAX_SEQS;
 constexpr size_t kStaticDecideBlocks = ((size_t)ULORL_STATIC_MAX_TOKENS + kDecideThreads - 1) / kDecideThreads;
 constexpr size_t kStaticScratchBytes = 256 + kStaticSeqBytes + sizeof(DecidePartial) * kStaticDecideBlocks;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
@@ -832,6 +882,39 @@ int ulorl_token_loss_decide_static(const ulorl_params_t* params, const float* lo
   if (cudaMemsetAsync(ws + pl.off_status, 0, 256, stream) != cudaSuccess) return ULORL_ERR_CUDA;
   return run_decide(params, pl, logp, entropy, old_logp, segment_version, advantages, seq_offsets, entropy_supplied,
                     grad_coef, flags, seq_entropy, loss, stats, ws, stream);
+}
+
+int ulorl_sequence_entropy_partials(const ulorl_params_t* params, const float* entropy, const int32_t* seq_offsets,
+                                    const int32_t* seq_ids, int32_t total_seqs, int64_t* table, void* workspace,
+                                    void* cuda_stream) {
+  int st = validate_params(params);
+  if (st != ULORL_OK) return st;
+  if (total_seqs < 0 || (total_seqs > 0 && !table)) return ULORL_ERR_INVALID_ARG;
+  if (!seq_ids && params->num_seqs > total_seqs) return ULORL_ERR_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (total_seqs > 0 && cudaMemsetAsync(table, 0, 2 * sizeof(int64_t) * (size_t)total_seqs, stream) != cudaSuccess)
+    return ULORL_ERR_CUDA;
+  if (params->T == 0 || params->num_seqs == 0) return ULORL_OK;
+  if (!entropy || !seq_offsets) return ULORL_ERR_INVALID_ARG;
+  static_assert(sizeof(long long) == sizeof(int64_t), "64-bit sums");
+  seq_entropy_partials_kernel<<<params->num_seqs, kSeqThreads, 0, stream>>>(
+      params->num_seqs, params->T, seq_offsets, entropy, seq_ids, total_seqs, reinterpret_cast<long long*>(table),
+      reinterpret_cast<int*>(workspace));
+  return check_launch();
+}
+
+int ulorl_sequence_entropy_combine(const int64_t* table, int32_t total_seqs, const int32_t* seq_ids, int32_t num_seqs,
+                                   float* seq_entropy, float* batch_entropy, void* cuda_stream) {
+  if (total_seqs < 0 || num_seqs < 0) return ULORL_ERR_INVALID_ARG;
+  if (!seq_ids && num_seqs > total_seqs) return ULORL_ERR_INVALID_ARG;
+  if (num_seqs == 0 && !batch_entropy) return ULORL_OK;
+  if (!table || (num_seqs > 0 && !seq_entropy)) return ULORL_ERR_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const int n = num_seqs > 0 ? num_seqs : 1;
+  seq_entropy_combine_kernel<<<(n + 127) / 128, 128, 0, stream>>>(num_seqs, seq_ids, total_seqs,
+                                                                 reinterpret_cast<const long long*>(table), seq_entropy,
+                                                                 batch_entropy);
+  return check_launch();
 }
 
 int ulorl_group_advantages(const float* rewards, int32_t num_responses, int32_t group_size, float* advantages,
@@ -948,7 +1031,7 @@ HostStepLayout host_step_layout(const ulorl_params_t* p) {
   L.loss = take(16);
   L.stats = take(sizeof(ulorl_stats_t));
   L.d_hidden = take(T * H * L.elem);
-  L.d_W = take(V * H * 4);
+  L.d_W = take(V * H * (p->dw_dtype == ULORL_BF16 ? 2 : 4));
   L.ws = take(make_plan(p).total);
   L.total = off;
   return L;
@@ -964,7 +1047,7 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
                                const int32_t* h_targets, const float* h_old_logp, const int32_t* h_segment_version,
                                const float* h_advantages, const int32_t* h_seq_offsets,
                                const float* h_entropy_supplied, float* h_logp, float* h_entropy, uint8_t* h_flags,
-                               float* h_seq_entropy, float* h_loss, void* h_stats, void* h_d_hidden, float* h_d_W,
+                               float* h_seq_entropy, float* h_loss, void* h_stats, void* h_d_hidden, void* h_d_W,
                                void* d_arena, size_t arena_bytes, void* cuda_stream) {
   int st = validate_params(params);
   if (st != ULORL_OK) return st;
@@ -1023,11 +1106,13 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
   // d_W rows go back slab by slab while the last panel is still being computed
   size_t n_slabs = 0;
   bool dw_by_slabs = false;
+  const size_t dw_elem = params->dw_dtype == ULORL_BF16 ? 2 : 4;
   if (pl.tensor && h_d_W) {
     hooks.after_dw_slab = [&](int v0, int v_rows) {
       cudaEvent_t e = hs->slab_event(n_slabs++);
       if (!e || !ok(cudaEventRecord(e, stream)) || !ok(cudaStreamWaitEvent(hs->out, e, 0)) ||
-          !ok(cudaMemcpyAsync(h_d_W + (size_t)v0 * H, a + L.d_W + (size_t)v0 * H * 4, (size_t)v_rows * H * 4,
+          !ok(cudaMemcpyAsync(static_cast<uint8_t*>(h_d_W) + (size_t)v0 * H * dw_elem,
+                              a + L.d_W + (size_t)v0 * H * dw_elem, (size_t)v_rows * H * dw_elem,
                               cudaMemcpyDeviceToHost, hs->out)))
         return (int)ULORL_ERR_CUDA;
       dw_by_slabs = true;
@@ -1055,11 +1140,11 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
     return ULORL_ERR_CUDA;
   st = bwd_impl(params, a + L.hidden, a + L.W, reinterpret_cast<const int32_t*>(a + L.targets),
                 reinterpret_cast<const float*>(a + L.lse), reinterpret_cast<const float*>(a + L.grad_coef), nullptr,
-                a + L.d_hidden, reinterpret_cast<float*>(a + L.d_W), a + L.ws, L.total - L.ws, stream, &hooks);
+                a + L.d_hidden, a + L.d_W, a + L.ws, L.total - L.ws, stream, &hooks);
   if (st != ULORL_OK) return st;
   // with compaction d_hidden is only final after the scatter at the end of the backward
   if (pl.compact && !ok(d2h(h_d_hidden, L.d_hidden, T * row_bytes))) return ULORL_ERR_CUDA;
-  if (!dw_by_slabs && !ok(d2h(h_d_W, L.d_W, V * H * 4))) return ULORL_ERR_CUDA;
+  if (!dw_by_slabs && !ok(d2h(h_d_W, L.d_W, V * H * dw_elem))) return ULORL_ERR_CUDA;
   // the caller's stream is done only when the outbound copies are
   if (!ok(cudaEventRecord(hs->out_done, hs->out)) || !ok(cudaStreamWaitEvent(stream, hs->out_done, 0))) return ULORL_ERR_CUDA;
   return ULORL_OK;

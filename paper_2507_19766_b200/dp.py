@@ -8,10 +8,47 @@ initialised with (NCCL over NVLink on GPUs, gloo in the CPU tests).
 """
 from __future__ import annotations
 
-from typing import List, Sequence
+import os
+import socket
+import subprocess
+import sys
+from typing import List, Optional, Sequence
 
 import torch
 import torch.distributed as dist
+
+
+# ---------------------------------------------------------------------------------------------
+# Launch: one process per GPU on this node.
+# ---------------------------------------------------------------------------------------------
+
+def free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return int(s.getsockname()[1])
+
+
+def launch_ranks(script: str, argv: Sequence[str], world_size: int, port: Optional[int] = None,
+                 env: Optional[dict] = None) -> int:
+    """Run `script argv...` as `world_size` ranks on this node (torch.distributed.run, rendezvous on
+    127.0.0.1) and return the launcher's exit code.  The ranks read RANK / LOCAL_RANK / WORLD_SIZE /
+    MASTER_* from their environment."""
+    if world_size < 1:
+        raise ValueError("world_size must be at least 1")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={world_size}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port or free_port()), script, *argv]
+    return subprocess.run(cmd, env=dict(os.environ, **(env or {}))).returncode
+
+
+def world_from_env(expected: int) -> tuple:
+    """(world size, rank, local rank) from the launcher's environment, or None when this process was not
+    started by a launcher; raises if the launcher's world size is not the one asked for."""
+    if "WORLD_SIZE" not in os.environ:
+        return None
+    world = int(os.environ["WORLD_SIZE"])
+    if world != expected:
+        raise RuntimeError(f"launched with WORLD_SIZE={world} but {expected} ranks were asked for")
+    return world, int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0"))
 
 
 def shard_sequences(lengths: Sequence[int], world_size: int) -> List[List[int]]:
@@ -48,6 +85,36 @@ def reduce_step_outputs(d_W: torch.Tensor, loss: torch.Tensor, counters: torch.T
         dist.all_reduce(counters)
 
 
+class SlabAllReduce:
+    """Sum of d_W over ranks, slab by slab, under the tail of the backward.  An instance is passed as the
+    slab callback of the backward call (ulorl_token_loss_bwd_slabs): each time the launches that make rows
+    [first_row, first_row + rows) of d_W final have been queued it starts an asynchronous all-reduce of
+    those rows.  The collective orders itself behind the work queued so far on the current stream and runs
+    on the backend's own stream, so the kernels queued afterwards (the next slab, d_hidden) overlap with
+    it; finish() makes the current stream wait for every slab.  The result equals one all-reduce of the
+    whole array: every element is summed over the same ranks either way."""
+
+    def __init__(self, d_W: torch.Tensor, group=None):
+        self.d_W = d_W
+        self.group = group
+        self.works = []
+        self.slabs = []
+        self.active = dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1
+
+    def __call__(self, first_row: int, rows: int):
+        self.slabs.append((first_row, rows))
+        if self.active and rows > 0:
+            self.works.append(dist.all_reduce(self.d_W[first_row:first_row + rows], group=self.group, async_op=True))
+
+    def finish(self):
+        for w in self.works:
+            w.wait()
+        self.works = []
+        covered = sorted(self.slabs)
+        self.slabs = []
+        return covered
+
+
 # ---------------------------------------------------------------------------------------------
 # Token-range sharding: when one ultra-long response dominates the batch, whole sequences no longer
 # balance and a rank takes a contiguous range of tokens instead.  A sequence can then straddle ranks,
@@ -77,33 +144,17 @@ def local_sequence_pieces(seq_offsets: Sequence[int], lo: int, hi: int):
     return ids, offs
 
 
-def sequence_entropy_partials(piece_mean: torch.Tensor, piece_tokens: torch.Tensor, ids: Sequence[int],
-                              num_seqs: int) -> torch.Tensor:
-    """[num_seqs, 2] float64 (entropy sum, token count) of this rank's pieces, zero elsewhere.  piece_mean is
-    what the forward call reports per local sequence (its seq_entropy output), piece_tokens their lengths."""
-    acc = torch.zeros(num_seqs, 2, dtype=torch.float64, device=piece_mean.device)
-    idx = torch.as_tensor(list(ids), dtype=torch.int64, device=acc.device)
-    n = piece_tokens.to(torch.float64).to(acc.device)
-    acc[idx, 0] = piece_mean.to(torch.float64) * n
-    acc[idx, 1] = n
-    return acc
-
-
-def sequence_entropy_from_partials(acc: torch.Tensor, ids: Sequence[int]) -> torch.Tensor:
-    """Mean entropy (float32, the type the decision stage compares with sigma) of the sequences `ids` from
-    the summed partials."""
-    idx = torch.as_tensor(list(ids), dtype=torch.int64, device=acc.device)
-    return (acc[idx, 0] / acc[idx, 1]).to(torch.float32)
-
-
-def exchange_sequence_entropy(piece_mean: torch.Tensor, piece_tokens: torch.Tensor, ids: Sequence[int],
-                              num_seqs: int) -> torch.Tensor:
-    """Mean entropy per sequence over all ranks' pieces, returned for this rank's pieces: one all-reduce of
-    [num_seqs, 2] float64 between the forward call and the decision stage (ent_scope = supplied)."""
-    acc = sequence_entropy_partials(piece_mean, piece_tokens, ids, num_seqs)
+def all_reduce_sequence_entropy(table: torch.Tensor) -> torch.Tensor:
+    """Sum, in place and over all ranks, the int64 [num_seqs, 2] tables (entropy sum in units of 2^-34 nats,
+    token count) that ulorl_sequence_entropy_partials fills from each rank's pieces.  Integer addition is
+    exact, so every rank ends with the sums of the unsplit batch bit for bit; the means are then taken on the
+    device by ulorl_sequence_entropy_combine and go to the decision stage as ent_scope = supplied.  This is
+    the one exchange between the forward call and the decision stage that token-range sharding adds."""
+    if table.dtype != torch.int64:
+        raise TypeError("the table of per-sequence entropy sums is int64")
     if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
-        dist.all_reduce(acc)
-    return sequence_entropy_from_partials(acc, ids)
+        dist.all_reduce(table)
+    return table
 
 
 def step_entropy_gate(call_mean_entropy: Sequence[float], call_tokens: Sequence[int], device=None) -> float:

@@ -95,9 +95,19 @@ def _token_range_worker(rank, world, port, result_dir):
         tg, ol, sv = batch.targets.numpy(), batch.old_logp.numpy(), batch.segment_version.numpy()
         _, ent, _ = O.token_stats(h[rows], w, tg[rows], 1.0)
         ent32 = ent.astype(np.float32)
-        means = torch.tensor([ent32[loff[k]:loff[k + 1]].astype(np.float64).mean() for k in range(len(ids))])
-        cnts = torch.tensor(np.diff(loff))
-        gate = dp.exchange_sequence_entropy(means, cnts, ids, wl.S).numpy()
+        # the exchange format of the library, restated: per sequence (sum of the float32 entropies in units of
+        # 2^-34 nats as int64, token count); integer sums are exact, so the all-reduce reproduces the unsplit sums
+        to_fixed = lambda e: np.rint(e.astype(np.float64) * 2.0 ** 34).astype(np.int64)
+        table = torch.zeros(wl.S, 2, dtype=torch.int64)
+        for k, i in enumerate(ids):
+            table[i, 0] = int(to_fixed(ent32[loff[k]:loff[k + 1]]).sum())
+            table[i, 1] = int(loff[k + 1] - loff[k])
+        dp.all_reduce_sequence_entropy(table)
+        _, ent_all, _ = O.token_stats(h, w, tg, 1.0)
+        fixed_all = to_fixed(ent_all.astype(np.float32))
+        assert table[:, 0].tolist() == [int(fixed_all[off[i]:off[i + 1]].sum()) for i in range(wl.S)]
+        assert table[:, 1].tolist() == np.diff(off).tolist()
+        gate = (table[ids, 0].numpy().astype(np.float64) * 2.0 ** -34 / table[ids, 1].numpy()).astype(np.float32)
         # sigma between the sequences' mean entropies, so that the gate is open for some and shut for others
         full_fwd = O.forward(h, w, tg, ol, sv, batch.advantages.numpy(), off, O.OracleParams())
         hbar = np.sort(full_fwd["seq_entropy"])
@@ -130,4 +140,53 @@ def _token_range_worker(rank, world, port, result_dir):
 def test_token_range_sharding_with_entropy_exchange(tmp_path):
     port = _free_port()
     mp.spawn(_token_range_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    assert (tmp_path / "ok").exists()
+
+
+def test_launch_ranks_starts_the_world_it_is_asked_for(tmp_path):
+    """bench.py --gpus N starts its own ranks through dp.launch_ranks; here two CPU ranks."""
+    import sys
+    probe = os.path.join(os.path.dirname(os.path.abspath(__file__)), "rank_probe.py")
+    rc = dp.launch_ranks(probe, [str(tmp_path), "2"], 2)
+    assert rc == 0
+    for r in range(2):
+        world, local_rank, total = (tmp_path / f"rank{r}").read_text().split()
+        assert (int(world), int(local_rank), int(total)) == (2, r, 3)
+    # a launcher whose world differs from what the script was asked for is an error, not a silent 1-rank run
+    rc = dp.launch_ranks(probe, [str(tmp_path), "3"], 2)
+    assert rc != 0
+    os.environ.pop("WORLD_SIZE", None)
+    assert dp.world_from_env(4) is None
+
+
+def _slab_worker(rank, world, port, result_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        V, H = 1000, 24
+        for dtype, exact in ((torch.float64, True), (torch.float32, False)):
+            g = torch.Generator().manual_seed(100 + rank)
+            mine = torch.randn(V, H, generator=g, dtype=torch.float64).to(dtype)
+            one_shot = mine.clone()
+            dist.all_reduce(one_shot)
+            by_slab = mine.clone()
+            red = dp.SlabAllReduce(by_slab)
+            # the slab schedule of the backward: ascending, covering [0, V) once, last slab ragged
+            for v0 in range(0, V, 296):
+                red(v0, min(296, V - v0))
+            covered = red.finish()
+            assert covered == [(0, 296), (296, 296), (592, 296), (888, 112)]
+            if exact:
+                assert torch.equal(by_slab, one_shot)
+            else:
+                assert torch.allclose(by_slab, one_shot, rtol=1e-6, atol=0) and torch.equal(by_slab, one_shot)
+        if rank == 0:
+            open(os.path.join(result_dir, "ok"), "w").write("ok")
+    finally:
+        dist.destroy_process_group()
+
+
+def test_slab_wise_reduction_equals_the_one_shot_sum(tmp_path):
+    port = _free_port()
+    mp.spawn(_slab_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
     assert (tmp_path / "ok").exists()

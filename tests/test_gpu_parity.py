@@ -414,15 +414,120 @@ def test_compacted_backward_with_nothing_active_and_with_accumulation():
     assert rel_l2((dW - 1.0).cpu().numpy(), dW_ref.cpu().numpy()) <= 1e-4
 
 
+# --------------------------------------------------------------------------- bf16 d_W, d_W slab by slab
+@pytest.mark.parametrize("path,panel,compact", [("tensor", 0, False), ("tensor", 384, False), ("tensor", 384, True),
+                                                ("tensor_1cta", 384, False), ("simt", 384, False)])
+def test_bf16_dw_output_matches_the_oracle_and_the_rounded_f32_result(path, panel, compact):
+    """dw_dtype = bf16: the sum over tokens is still taken in float32 and rounded once when final, so the
+    result is the float32 d_W rounded to bf16 (bit for bit), and it keeps the gradient tolerance to the oracle."""
+    wl = synth.WORKLOADS["small"].scaled(T=700, S=5, H=328, V=3001, lengths="lognormal:100:400",
+                                         segment_len=64, planted=0.3, beta_planted=(80.0, 160.0),
+                                         mpt_mode="dynamic", entropy_target=6.0)
+    batch = synth.make_batch(wl, seed=5)
+    import dataclasses
+    gp32, op = both_params(batch, kernel_path=path, bwd_panel_tokens=panel, compact_rows=compact)
+    gp16 = dataclasses.replace(gp32, dw_dtype="bf16")
+    assert B.workspace_bytes(gp16) >= B.workspace_bytes(gp32) + 4 * wl.V * wl.H
+    out, dH32, dW32 = gpu_fwd_bwd(batch, gp32)
+    _, dH16, dW16 = gpu_fwd_bwd(batch, gp16)
+    assert dW16.dtype == torch.bfloat16 and torch.equal(dH16, dH32)
+    assert torch.equal(dW16, dW32.to(torch.bfloat16))
+    oi = oracle_inputs(batch)
+    _, dW_ref = O.backward(oi["hidden"], oi["W"], oi["targets"], out.grad_coef.cpu().numpy().astype(np.float64))
+    assert rel_l2(dW16.float().cpu().numpy(), dW_ref) <= TOL_GRAD
+    # accumulation into the caller's bf16 array: old + sum, rounded once
+    gp_acc = dataclasses.replace(gp16, dw_accumulate=True)
+    b = batch.to(DEV)
+    ws = B.alloc_workspace(gp_acc, DEV)
+    old = (torch.randn(wl.V, wl.H, device=DEV) * dW32.abs().mean()).to(torch.bfloat16)
+    dW = old.clone()
+    B.token_loss_bwd(gp_acc, b.hidden, b.W, b.targets, out.lse, out.grad_coef, d_W=dW, workspace=ws)
+    assert torch.equal(dW, (old.float() + dW32).to(torch.bfloat16))
+
+
+@pytest.mark.parametrize("path,V,panel,dw_dtype", [("tensor", 40000, 512, "f32"), ("tensor", 40000, 512, "bf16"),
+                                                   ("tensor", 2500, 0, "f32"), ("simt", 2500, 256, "f32")])
+def test_backward_reports_dw_slab_by_slab(path, V, panel, dw_dtype):
+    """ulorl_token_loss_bwd_slabs: the callback sees ascending slabs that cover [0, V) once, the rows it is told
+    about are final when the work queued before the callback has run (an event recorded inside the callback
+    orders a copy on a second stream), and the results are those of the plain backward bit for bit."""
+    wl = synth.WORKLOADS["small"].scaled(T=900, S=4, H=256, V=V, lengths="tiny", planted=0.3,
+                                         beta_planted=(100.0, 200.0), mpt_mode="always")
+    batch = synth.make_batch(wl, seed=41)
+    gp, _ = both_params(batch, kernel_path=path, bwd_panel_tokens=panel)
+    import dataclasses
+    gp = dataclasses.replace(gp, dw_dtype=dw_dtype)
+    out, dH, dW = gpu_fwd_bwd(batch, gp)
+    b = batch.to(DEV)
+    ws = B.alloc_workspace(gp, DEV)
+    dW2 = torch.full((wl.V, wl.H), 7.0, dtype=gp.dw_torch_dtype, device=DEV)
+    copy = torch.zeros_like(dW2)
+    side = torch.cuda.Stream()
+    slabs = []
+
+    def on_slab(first_row, rows):
+        slabs.append((first_row, rows))
+        ev = torch.cuda.Event()
+        ev.record()                                   # behind the launches that make these rows final
+        side.wait_event(ev)
+        with torch.cuda.stream(side):
+            copy[first_row:first_row + rows].copy_(dW2[first_row:first_row + rows], non_blocking=True)
+
+    dH2, _ = B.token_loss_bwd(gp, b.hidden, b.W, b.targets, out.lse, out.grad_coef, d_W=dW2, workspace=ws,
+                              on_dw_slab=on_slab)
+    torch.cuda.synchronize()
+    assert slabs[0][0] == 0 and sum(r for _, r in slabs) == wl.V
+    assert all(slabs[i][0] + slabs[i][1] == slabs[i + 1][0] for i in range(len(slabs) - 1))
+    if path == "tensor" and V == 40000:
+        assert len(slabs) > 1                          # several waves of vocabulary row tiles
+    assert torch.equal(dW2, dW) and torch.equal(dH2, dH) and torch.equal(copy, dW)
+    # an exception raised inside the callback stops the pass and reaches the caller
+    def boom(first_row, rows):
+        raise ValueError("stop here")
+    with pytest.raises(ValueError, match="stop here"):
+        B.token_loss_bwd(gp, b.hidden, b.W, b.targets, out.lse, out.grad_coef, d_W=dW2, workspace=ws, on_dw_slab=boom)
+    torch.cuda.synchronize()
+
+
+def test_sequence_entropy_tables_edge_cases():
+    """The exact per-sequence entropy tables: identity ids, pieces of one sequence inside one call, ids out of
+    range reported and skipped, and the means of an unsplit call reproduced."""
+    rng = np.random.default_rng(8)
+    T, S = 3000, 5
+    ent = torch.from_numpy((rng.random(T) * 3.0).astype(np.float32)).to(DEV)
+    off = torch.tensor([0, 10, 10, 1500, 2999, 3000], dtype=torch.int32, device=DEV)     # one empty sequence
+    p = B.Params(T=T, H=8, V=16, num_seqs=S, dtype="f32")
+    table = B.sequence_entropy_partials(p, ent, off, None, S)
+    fixed = np.rint(ent.cpu().numpy().astype(np.float64) * 2.0 ** 34).astype(np.int64)
+    o = off.cpu().numpy()
+    assert table[:, 0].cpu().tolist() == [int(fixed[o[i]:o[i + 1]].sum()) for i in range(S)]
+    assert table[:, 1].cpu().tolist() == np.diff(o).tolist()
+    means, batch = B.sequence_entropy_combine(table, None, S, want_batch=True)
+    dec = B.token_loss_decide(p, ent.clone(), ent, ent, None, torch.ones(S, device=DEV), off)
+    assert torch.equal(means, dec.seq_entropy[:S]) and float(means[1]) == 0.0
+    assert float(batch[0]) == dec.stats_host()["mean_entropy"]
+    # two pieces of sequence 3 and one of sequence 0 in one call of a 6-sequence step; id 9 is out of range
+    ids = torch.tensor([3, 0, 3, 9, 5], dtype=torch.int32, device=DEV)
+    ws = torch.zeros(256, dtype=torch.uint8, device=DEV)
+    t2 = B.sequence_entropy_partials(p, ent, off, ids, 6, workspace=ws)
+    assert t2[3].cpu().tolist() == [int(fixed[0:10].sum() + fixed[10:1500].sum()), 1500]
+    assert t2[0].cpu().tolist() == [0, 0] and t2[5].cpu().tolist() == [int(fixed[2999]), 1]
+    assert t2[[1, 2, 4]].abs().sum().item() == 0
+    assert B.check_status(ws) == -1
+
+
 # --------------------------------------------------------------------------- host-buffer step, timing aid, bad offsets
-@pytest.mark.parametrize("V,panel,compact", [(2500, 0, False), (40000, 512, False), (40000, 512, True)])
-def test_host_buffer_step_matches_device_calls(V, panel, compact):
+@pytest.mark.parametrize("V,panel,compact,dw_dtype", [(2500, 0, False, "f32"), (40000, 512, False, "f32"),
+                                                      (40000, 512, True, "f32"), (40000, 512, False, "bf16")])
+def test_host_buffer_step_matches_device_calls(V, panel, compact, dw_dtype):
     # the second case has two backward panels and a vocabulary of several d_W slabs: on the last panel the
     # host-buffer step computes d_W slab by slab, ahead of d_hidden, and copies each slab out as it is done
     wl = synth.WORKLOADS["small"].scaled(T=900, S=4, H=256, V=V, lengths="tiny", planted=0.3,
                                          beta_planted=(100.0, 200.0), mpt_mode="always")
     batch = synth.make_batch(wl, seed=41)
     gp, _ = both_params(batch, bwd_panel_tokens=panel, compact_rows=compact)
+    import dataclasses
+    gp = dataclasses.replace(gp, dw_dtype=dw_dtype)
     out, dH, dW = gpu_fwd_bwd(batch, gp)
     arena = torch.empty(B.host_step_arena_bytes(gp), dtype=torch.uint8, device=DEV)
     pin = lambda t: t.contiguous().pin_memory()
@@ -430,7 +535,7 @@ def test_host_buffer_step_matches_device_calls(V, panel, compact):
               flags=torch.empty(wl.T, dtype=torch.uint8).pin_memory(), seq_entropy=torch.empty(wl.S).pin_memory(),
               loss=torch.empty(1).pin_memory(), stats=torch.empty(out.stats.numel(), dtype=torch.uint8).pin_memory(),
               d_hidden=torch.empty(wl.T, wl.H, dtype=torch.bfloat16).pin_memory(),
-              d_W=torch.empty(wl.V, wl.H).pin_memory())
+              d_W=torch.empty(wl.V, wl.H, dtype=gp.dw_torch_dtype).pin_memory())
     for _ in range(2):                                   # the arena is reusable across calls
         B.token_loss_step_host(gp, arena, pin(batch.hidden), pin(batch.W), pin(batch.targets), pin(batch.old_logp),
                                pin(batch.segment_version), pin(batch.advantages), pin(batch.seq_offsets), **ho)
@@ -495,59 +600,72 @@ def test_group_advantages_match_the_oracle():
 
 def test_token_range_split_with_entropy_exchange_matches_the_unsplit_batch():
     """Two token ranges of one batch, run one after the other as two ranks would run them: forward on each
-    range, per-sequence (entropy sum, count) partials summed, decision stage with the means supplied,
-    backward accumulating into one d_W.  Flags, loss and gradients equal the unsplit run's."""
+    range, the library's exact per-sequence (entropy sum, count) tables added as an int64 all-reduce would add
+    them, the means taken on the device, decision stage with the means supplied, backward accumulating into
+    one d_W.  The mean entropy of every sequence is the unsplit run's bit for bit, so with sigma one float32
+    step above, at, and one step below a split sequence's H-bar the flags, loss and gradients equal the
+    unsplit run's."""
     import dataclasses
     from paper_2507_19766_b200 import dp
     wl = synth.WORKLOADS["small"].scaled(T=1500, S=4, H=128, V=1500, lengths="fixed:700,400,300,100", planted=0.6,
                                          beta_planted=(200.0, 450.0), mpt_mode="dynamic", adv="bern:0.5:3")
     batch = synth.make_batch(wl, seed=26)
-    gp, op = both_params(batch)
+    gp0, op0 = both_params(batch)
     oi = oracle_inputs(batch)
     ref = O.forward(oi["hidden"], oi["W"], oi["targets"], oi["old_logp"], oi["segment_version"], oi["advantages"],
-                    oi["seq_offsets"], op)
-    hbar = np.sort(ref["seq_entropy"])
-    sigma = float(0.5 * (hbar[1] + hbar[2]))                    # gate open for two sequences, shut for two
-    assert min(hbar[2] - sigma, sigma - hbar[1]) > 10 * TOL_LOGP
-    gp, op = both_params(batch, entropy_target=sigma)
-    full, dH_full, dW_full = gpu_fwd_bwd(batch, gp)
+                    oi["seq_offsets"], op0)
     b = batch.to(DEV)
     off = batch.seq_offsets.numpy()
     ranges = dp.shard_token_ranges(wl.T, 2, align=256)
-    assert ranges == [(0, 768), (768, 1500)]                   # sequences 0 and 1 are both split
-    pieces, partial = [], torch.zeros(wl.S, 2, dtype=torch.float64, device=DEV)
-    for lo, hi in ranges:
-        ids, loff = dp.local_sequence_pieces(off, lo, hi)
-        lp = dataclasses.replace(gp, T=hi - lo, num_seqs=len(ids), norm_tokens=wl.T, ent_scope="supplied",
-                                 dw_accumulate=True)
-        loff_t = torch.tensor(loff, dtype=torch.int32, device=DEV)
-        adv = b.advantages[torch.tensor(ids, device=DEV)].contiguous()
-        dummy = torch.zeros(len(ids), dtype=torch.float32, device=DEV)
-        sl = slice(lo, hi)
-        f = B.token_loss_fwd(lp, b.hidden[sl], b.W, b.targets[sl], b.old_logp[sl], b.segment_version[sl], adv, loff_t,
-                             entropy_supplied=dummy)
-        cnt = torch.tensor(np.diff(loff), device=DEV)
-        partial += dp.sequence_entropy_partials(f.seq_entropy[:len(ids)], cnt, ids, wl.S)
-        pieces.append((sl, ids, lp, loff_t, adv, f))
-    dW = torch.zeros(wl.V, wl.H, dtype=torch.float32, device=DEV)
-    dH = torch.empty_like(b.hidden)
-    loss, flags = 0.0, np.zeros(wl.T, dtype=np.uint8)
-    for sl, ids, lp, loff_t, adv, f in pieces:
-        gate = dp.sequence_entropy_from_partials(partial, ids)
-        d = B.token_loss_decide(lp, f.logp, f.entropy, b.old_logp[sl], b.segment_version[sl], adv, loff_t,
-                                entropy_supplied=gate)
-        B.token_loss_bwd(lp, b.hidden[sl], b.W, b.targets[sl], f.lse, d.grad_coef, d_hidden=dH[sl], d_W=dW)
-        loss += float(d.loss.cpu()[0])
-        flags[sl] = d.flags.cpu().numpy()
-    torch.cuda.synchronize()
-    gate_all = dp.sequence_entropy_from_partials(partial, range(wl.S)).cpu().numpy()
-    assert np.abs(gate_all - ref["seq_entropy"]).max() <= TOL_LOGP
-    assert np.array_equal(flags, full.flags.cpu().numpy())
-    masked = (flags & O.FLAG_MASKED) != 0
-    assert 0 < masked.sum() < ((flags & O.FLAG_MPT) != 0).sum()
-    assert abs(loss - float(full.loss.cpu()[0])) <= 1e-5 * max(1e-3, abs(loss))
-    assert torch.equal(dH, dH_full)                            # rows are independent of the split
-    assert rel_l2(dW.cpu().numpy(), dW_full.cpu().numpy()) <= 1e-4
+    assert ranges == [(0, 768), (768, 1500)]                   # sequence 1 (tokens 700..1100) is split
+    base, _, _ = gpu_fwd_bwd(batch, gp0)
+    hbar = base.seq_entropy.cpu().numpy()[:wl.S].astype(np.float32)
+    assert np.abs(hbar - ref["seq_entropy"]).max() <= TOL_LOGP
+    split_seq = 1
+    up, down = np.nextafter(hbar[split_seq], np.float32(np.inf)), np.nextafter(hbar[split_seq], np.float32(-np.inf))
+    masked_counts = []
+    for sigma in (float(up), float(hbar[split_seq]), float(down)):
+        gp, _ = both_params(batch, entropy_target=sigma)
+        full, dH_full, dW_full = gpu_fwd_bwd(batch, gp)
+        pieces = []
+        table = torch.zeros(wl.S, 2, dtype=torch.int64, device=DEV)
+        for lo, hi in ranges:
+            ids, loff = dp.local_sequence_pieces(off, lo, hi)
+            lp = dataclasses.replace(gp, T=hi - lo, num_seqs=len(ids), norm_tokens=wl.T, ent_scope="supplied",
+                                     dw_accumulate=True)
+            loff_t = torch.tensor(loff, dtype=torch.int32, device=DEV)
+            ids_t = torch.tensor(ids, dtype=torch.int32, device=DEV)
+            adv = b.advantages[ids_t.long()].contiguous()
+            dummy = torch.zeros(len(ids), dtype=torch.float32, device=DEV)
+            sl = slice(lo, hi)
+            f = B.token_loss_fwd(lp, b.hidden[sl], b.W, b.targets[sl], b.old_logp[sl], b.segment_version[sl], adv,
+                                 loff_t, entropy_supplied=dummy)
+            table += B.sequence_entropy_partials(lp, f.entropy, loff_t, ids_t, wl.S)   # what the all-reduce sums
+            pieces.append((sl, ids_t, lp, loff_t, adv, f))
+        dp.all_reduce_sequence_entropy(table)                   # no process group here: returns the table as is
+        dW = torch.zeros(wl.V, wl.H, dtype=torch.float32, device=DEV)
+        dH = torch.empty_like(b.hidden)
+        loss, flags = 0.0, np.zeros(wl.T, dtype=np.uint8)
+        for sl, ids_t, lp, loff_t, adv, f in pieces:
+            gate = B.sequence_entropy_combine(table, ids_t, ids_t.numel())
+            d = B.token_loss_decide(lp, f.logp, f.entropy, b.old_logp[sl], b.segment_version[sl], adv, loff_t,
+                                    entropy_supplied=gate)
+            B.token_loss_bwd(lp, b.hidden[sl], b.W, b.targets[sl], f.lse, d.grad_coef, d_hidden=dH[sl], d_W=dW)
+            loss += float(d.loss.cpu()[0])
+            flags[sl] = d.flags.cpu().numpy()
+        torch.cuda.synchronize()
+        gate_all, batch_mean = B.sequence_entropy_combine(table, None, wl.S, want_batch=True)
+        assert torch.equal(gate_all, full.seq_entropy[:wl.S])      # bit for bit, split or not
+        assert float(batch_mean.cpu()[0]) == full.stats_host()["mean_entropy"]
+        assert table[:, 1].cpu().tolist() == np.diff(off).tolist()
+        assert np.array_equal(flags, full.flags.cpu().numpy())
+        assert abs(loss - float(full.loss.cpu()[0])) <= 1e-5 * max(1e-3, abs(loss))
+        assert torch.equal(dH, dH_full)                            # rows are independent of the split
+        assert rel_l2(dW.cpu().numpy(), dW_full.cpu().numpy()) <= 1e-4
+        seq_of = np.repeat(np.arange(wl.S), np.diff(off))
+        masked_counts.append(int(((flags & O.FLAG_MASKED) != 0)[seq_of == split_seq].sum()))
+    # one float32 step of sigma across the split sequence's H-bar opens and shuts its gate (H-bar < sigma, strict)
+    assert masked_counts[0] > 0 and masked_counts[1] == 0 and masked_counts[2] == 0
 
 
 @pytest.mark.parametrize("path,norm_seqs", [("tensor", 0), ("simt", 9)])
