@@ -5,7 +5,7 @@ from __future__ import annotations
 import numpy as np
 
 from oracle import ulorl_oracle as O
-from paper_2507_19766_b200 import synth
+from workloads import synth
 from paper_2507_19766_b200.binding import Params
 
 # tolerances of the parity contract

@@ -36,7 +36,7 @@ def _worker(rank, world, port, result_dir):
     dist.init_process_group("gloo", rank=rank, world_size=world)
     try:
         from oracle import ulorl_oracle as O
-        from paper_2507_19766_b200 import synth
+        from workloads import synth
         wl = synth.WORKLOADS["small"].scaled(T=96, S=6, H=16, V=64, lengths="lognormal:16:40", segment_len=8,
                                              planted=0.3, beta_planted=(30.0, 60.0), mpt_mode="always")
         batch = synth.make_batch(wl, seed=11)          # every rank builds the same global batch
@@ -81,7 +81,7 @@ def _token_range_worker(rank, world, port, result_dir):
     dist.init_process_group("gloo", rank=rank, world_size=world)
     try:
         from oracle import ulorl_oracle as O
-        from paper_2507_19766_b200 import synth
+        from workloads import synth
         wl = synth.WORKLOADS["small"].scaled(T=90, S=3, H=16, V=64, lengths="fixed:50,25,15", segment_len=8,
                                              planted=0.6, beta_planted=(1500.0, 4000.0), mpt_mode="dynamic")   # H = 16: |W_y|^2 is tiny
         batch = synth.make_batch(wl, seed=14)

@@ -9,7 +9,7 @@ import torch
 
 from oracle import ulorl_oracle as O
 from paper_2507_19766_b200 import binding as B
-from paper_2507_19766_b200 import synth
+from workloads import synth
 from tests.helpers import TOL_GRAD, TOL_LOGP, both_params, rel_l2
 
 pytestmark = pytest.mark.gpu
@@ -41,7 +41,7 @@ def stratified_rows(batch, n_random=160, seed=0):
     return rows
 
 
-@pytest.mark.parametrize("name", ["ultra", "qwen", "mixed"])
+@pytest.mark.parametrize("name", ["ultra", "ultra_open", "qwen", "mixed"])
 def test_full_size_workload_against_sampled_oracle(name):
     wl = synth.WORKLOADS[name]
     batch = synth.make_batch(wl, device=DEV)
@@ -87,6 +87,9 @@ def test_full_size_workload_against_sampled_oracle(name):
     assert st["n_clip_low"] == int(((flags & O.FLAG_CLIP_LOW) != 0).sum())
     if name == "ultra":        # the recipe puts the mean entropy below sigma: the dynamic gate is open
         assert seq_ent[0] < wl.entropy_target and st["n_masked"] > wl.T // 2 and st["n_active"] > wl.T // 20
+    if name == "ultra_open":   # weaker plants: mean entropy above sigma, the gate stays shut, MPTs are not masked
+        assert seq_ent[0] > wl.entropy_target and st["n_masked"] == 0 and st["n_mpt"] > wl.T // 4
+        assert st["n_active"] > wl.T // 2
     if name == "mixed":
         assert st["n_clip_high"] == 0 and st["n_clip_low"] == 0
     if name == "qwen":         # static masking: planted targets of positive sequences are masked

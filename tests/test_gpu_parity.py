@@ -7,7 +7,7 @@ import torch
 
 from oracle import ulorl_oracle as O
 from paper_2507_19766_b200 import binding as B
-from paper_2507_19766_b200 import synth
+from workloads import synth
 from tests.helpers import TOL_GRAD, TOL_LOGP, TOL_LOSS, both_params, near_threshold, oracle_inputs, rel_l2
 
 pytestmark = pytest.mark.gpu
@@ -685,3 +685,38 @@ def test_per_sample_normalisation_matches_the_oracle(path, norm_seqs):
     G = norm_seqs if norm_seqs else wl.S
     scale = np.repeat(wl.T / (G * lens.astype(np.float64)), lens)          # (1/(G|o_i|)) / (1/T)
     assert np.allclose(out.grad_coef.cpu().numpy(), out_t.grad_coef.cpu().numpy() * scale, rtol=1e-6, atol=1e-12)
+
+
+def test_slab_wise_all_reduce_on_a_one_rank_nccl_group():
+    """The data-parallel step as bench.py runs it, on a process group of one rank: the backward hands d_W to
+    dp.SlabAllReduce slab by slab, each slab is all-reduced asynchronously on the backend's stream behind the
+    launches that made it final, and finish() joins them.  With one rank the sum is the rank's own d_W, which
+    must be the plain backward's bit for bit; what this exercises is the ordering between the compute stream
+    and the collective's stream."""
+    import torch.distributed as dist
+    from paper_2507_19766_b200 import dp
+    wl = synth.WORKLOADS["small"].scaled(T=900, S=4, H=256, V=40000, lengths="tiny", planted=0.3,
+                                         beta_planted=(100.0, 200.0), mpt_mode="always")
+    batch = synth.make_batch(wl, seed=41)
+    gp, _ = both_params(batch, bwd_panel_tokens=512)
+    out, dH, dW = gpu_fwd_bwd(batch, gp)
+    b = batch.to(DEV)
+    ws = B.alloc_workspace(gp, DEV)
+    created = not dist.is_initialized()
+    if created:
+        dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{dp.free_port()}", rank=0, world_size=1,
+                                device_id=torch.device(DEV))
+    try:
+        dW2 = torch.full((wl.V, wl.H), 3.0, device=DEV)
+        red = dp.SlabAllReduce(dW2)
+        red.active = True                    # a one-rank group would otherwise skip the collective
+        dH2, _ = B.token_loss_bwd(gp, b.hidden, b.W, b.targets, out.lse, out.grad_coef, d_W=dW2, workspace=ws,
+                                  on_dw_slab=red)
+        assert len(red.works) > 1
+        covered = red.finish()
+        torch.cuda.synchronize()
+        assert covered[0][0] == 0 and sum(r for _, r in covered) == wl.V
+        assert torch.equal(dW2, dW) and torch.equal(dH2, dH)
+    finally:
+        if created:
+            dist.destroy_process_group()

@@ -2,7 +2,7 @@
 import numpy as np
 import pytest
 
-from paper_2507_19766_b200 import synth
+from workloads import synth
 
 
 def test_batches_are_a_pure_function_of_workload_and_seed():

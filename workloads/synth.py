@@ -9,9 +9,16 @@ Eq. 8), 0/1 rewards turned into group-normalised advantages (Eq. 4), and a share
 sharply peaked rows so that well-mastered positive tokens (Eq. 9) actually occur.
 
 Random numbers come from NumPy's counter-based Philox generator; a batch is a pure
-function of (workload, seed).  The old log-probs a rollout engine would have recorded
-are imitated by `rollout_logp` (library matmul + logsumexp in float32) plus per-segment
-noise; a caller may instead hand in log-probs from elsewhere as the noise's base.
+function of (workload, seed).
+
+Two recipes imitate what the parts of the training loop upstream of the policy update hand
+over; they are input recipes, not implementations anyone is checked against.  `rollout_logp`
+stands in for the rollout engine's record of the log-prob of each generated token (library
+matmul + logsumexp in float32) and for its sampler (inverse-CDF draw from the row softmax with
+supplied uniforms); per-segment noise is added on top, and a caller may hand in log-probs from
+elsewhere as the noise's base.  `_advantages` stands in for the reward model followed by the
+group normalisation of Eq. 4 (library mean and standard deviation).  No expected value of any
+test comes from either: the oracle and the CUDA path both just receive the arrays.
 """
 from __future__ import annotations
 
