@@ -285,11 +285,11 @@ int ulorl_kernel_timing_end(float* total_ms, int64_t* launches);
  * h_d_W[V,H] (params->dw_dtype).  d_arena is DEVICE memory of at least ulorl_host_step_arena_bytes(params)
  * bytes, owned by the caller and reusable across calls; it holds the device copies, the outputs
  * and the workspace.  Asynchronous on cuda_stream: synchronise the stream before reading outputs
- * or reusing the host buffers.  Copies are overlapped with the passes: hidden states arrive in
- * panel-sized chunks on an inbound copy stream while the statistics kernel already runs on the
- * chunks that have landed, and the d_hidden rows of each backward panel leave on an outbound copy
- * stream while the next panel is computed (W has to be there first and d_W is only final at the
- * end, so those two copies are not hidden).  The two copy streams and their events are created on
+ * or reusing the host buffers.  Copies are overlapped with the passes: a first chunk of hidden states
+ * arrives, then W in slabs of vocabulary rows while the statistics kernel already sweeps that chunk
+ * against the slabs that have landed, then the other chunks while it runs on those before them; the
+ * d_hidden rows of each backward panel leave on an outbound copy stream while the next panel is
+ * computed, and on the last panel d_W is computed first and leaves slab by slab under the rest.  The two copy streams and their events are created on
  * the first call and kept for the life of the process; cuda_stream waits for both before the call's
  * work on it is complete.
  */

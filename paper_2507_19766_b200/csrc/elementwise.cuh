@@ -12,11 +12,12 @@ namespace ulorl {
 // a = hidden . W[v], s = sum_v exp(kappa (a_v - m)), u = sum_v exp(kappa (a_v - m)) (a_v - m).
 //   lse = kappa m* + ln s*,  logp = kappa a_y - lse,  Hent = ln s* - kappa u* / s*.
 // ------------------------------------------------------------------------------------------
-__global__ void merge_splits_kernel(int T, int n_split, float kappa, const float4* __restrict__ partials,
-                                    const float* __restrict__ acc_y, float* __restrict__ logp,
-                                    float* __restrict__ entropy, float* __restrict__ lse) {
-  const int t = blockIdx.x * blockDim.x + threadIdx.x;
-  if (t >= T) return;
+// Tokens [t_begin, t_end) of a batch of T; ranges of tokens may have been given different split counts.
+__global__ void merge_splits_kernel(int T, int t_begin, int t_end, int n_split, float kappa,
+                                    const float4* __restrict__ partials, const float* __restrict__ acc_y,
+                                    float* __restrict__ logp, float* __restrict__ entropy, float* __restrict__ lse) {
+  const int t = t_begin + blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= t_end) return;
   float m = -INFINITY;
   for (int k = 0; k < n_split; ++k) m = fmaxf(m, partials[(size_t)k * T + t].x);
   float s = 0.f, u = 0.f;

@@ -25,6 +25,7 @@ constexpr int kMaxDevices = 64;            // per-device set-up tables
 constexpr int kFallbackSMs = 148;         // B200; used for the plan when no device can be asked
 constexpr int kDefaultPanelTensor = 16384;       // single-CTA kernels
 constexpr int kDefaultPanelSimt = 1024;
+constexpr int kFirstChunkSlots = 16;      // partial slots a first chunk may use when W arrives in slabs (host-buffer step)
 constexpr int kRasterGroup = 16;          // dz: row tiles per raster group (m fastest inside a group)
 constexpr int kGradRasterGroup = 1;       // d_hidden, d_W: column blocks of one row tile run side by side, so its A stream is read once
 
@@ -59,6 +60,7 @@ struct Plan {
   int cta;                // CTAs per tcgen05.mma: 2 (a CTA pair per 256 x 256 tile) or 1 (ULORL_PATH_TENSOR_1CTA)
   int sms;                // multiprocessors the persistent kernels are spread over
   int n_split, tiles_per_split;
+  int partial_slots;      // slots per token in the softmax partials: n_split, or more for a first chunk swept slab by slab
   int panel_tokens;
   size_t dz_ld;           // leading dimension of the dz panel (elements)
   size_t off_status, off_batch_mean, off_seq_sum, off_partials, off_acc_y, off_decide, off_dz, total;
@@ -157,7 +159,8 @@ static Plan make_plan(const ulorl_params_t* p) {
   pl.off_status = off;      off += 256;
   pl.off_batch_mean = pl.off_status + 16;
   pl.off_seq_sum = off;     off = align_up(off + sizeof(long long) * (size_t)(p->num_seqs > 0 ? p->num_seqs : 1), 256);
-  pl.off_partials = off;    off = align_up(off + sizeof(float4) * (size_t)pl.n_split * (size_t)(T > 0 ? T : 1), 256);
+  pl.partial_slots = pl.tensor ? std::max(pl.n_split, std::min(kFirstChunkSlots, n_tiles)) : pl.n_split;
+  pl.off_partials = off;    off = align_up(off + sizeof(float4) * (size_t)pl.partial_slots * (size_t)(T > 0 ? T : 1), 256);
   pl.off_acc_y = off;       off = align_up(off + sizeof(float) * (size_t)(T > 0 ? T : 1), 256);
   pl.off_decide = off;      off = align_up(off + sizeof(DecidePartial) * (size_t)(pl.decide_blocks > 0 ? pl.decide_blocks : 1), 1024);
   pl.off_dz = off;          off = align_up(off + (size_t)panel * pl.dz_ld * (pl.tensor ? 2 : 4), 1024);
@@ -410,7 +413,13 @@ static int empty_forward(void* workspace, size_t workspace_bytes, float* loss, v
 // launches the statistics kernel once per chunk of tokens (all at once without hooks), the backward
 // reports every token panel whose d_hidden rows are final.
 struct StepHooks {
-  int chunk_tokens = 0;
+  // Forward, tensor path: the statistics kernel is launched once per chunk of tokens; chunk c covers tokens
+  // [chunk_starts[c], chunk_starts[c + 1]) (the last one runs to T; empty = one chunk).  With w_slabs > 1 the
+  // FIRST chunk is swept in w_slabs launches, one per range of vocabulary tiles, and before_w_slab(k, first row,
+  // rows) is called before launch k: W may still be arriving while the chunk's first launches run.
+  std::vector<int> chunk_starts;
+  int w_slabs = 0;
+  std::function<int(int, int, int)> before_w_slab;
   std::function<int(int, int)> before_stats_chunk;    // (first token, tokens) -> status
   std::function<int(int, int)> after_dhidden_panel;   // (first token, tokens) -> status; dense backward only
   // Tensor path: when set, the last panel computes d_W before d_hidden and in slabs of vocabulary rows,
@@ -507,20 +516,19 @@ static int fwd_impl(const ulorl_params_t* params, const void* hidden, const void
     st = make_map_bf16(&map_b, W, (uint64_t)V, (uint64_t)H, (uint64_t)H, kBK, kBN / pl.cta);
     if (st != ULORL_OK) return st;
     const int tile_m = kBM * pl.cta;
-    int chunk = (hooks && hooks->chunk_tokens > 0) ? hooks->chunk_tokens : T;
-    chunk = (chunk + tile_m - 1) / tile_m * tile_m;
-    for (int t0 = 0; t0 < T; t0 += chunk) {
-      const int rows = (T - t0) < chunk ? (T - t0) : chunk;
-      if (hooks && hooks->before_stats_chunk) {
-        st = hooks->before_stats_chunk(t0, rows);
-        if (st != ULORL_OK) return st;
-      }
+    const int n_tiles = (V + kBN - 1) / kBN;
+    std::vector<int> starts = (hooks && !hooks->chunk_starts.empty()) ? hooks->chunk_starts : std::vector<int>{0};
+    starts.push_back(T);
+    auto launch_stats = [&](int t0, int rows, int n_split, int tiles_per_split, int tile_base, int tile_end,
+                            int split_base) -> int {
       UmmaArgs a{};
       a.M = rows; a.N = V; a.K = H;
       a.m_tiles = (rows + tile_m - 1) / tile_m;
-      a.n_tiles = (V + kBN - 1) / kBN;
-      a.n_split = pl.n_split;
-      a.tiles_per_split = pl.tiles_per_split;
+      a.n_tiles = tile_end;
+      a.n_split = n_split;
+      a.tiles_per_split = tiles_per_split;
+      a.tile_base = tile_base;
+      a.split_base = split_base;
       a.a_mn0 = t0;
       a.row0 = t0;
       a.kappa = kappa;
@@ -529,8 +537,47 @@ static int fwd_impl(const ulorl_params_t* params, const void* hidden, const void
       a.acc_y = acc_y;
       a.T_total = T;
       a.status = status;
-      st = launch_umma<kModeStats>(pl, map_a, map_b, map_a, a, stream);
-      if (st != ULORL_OK) return st;
+      return launch_umma<kModeStats>(pl, map_a, map_b, map_a, a, stream);
+    };
+    // tokens [0, slab_rows_end) get their statistics from w_slabs launches over vocabulary ranges
+    int slab_tokens = 0, slab_slots = 0;
+    for (size_t c = 0; c + 1 < starts.size(); ++c) {
+      const int t0 = starts[c], rows = starts[c + 1] - starts[c];
+      if (rows <= 0 || t0 % tile_m != 0) return ULORL_ERR_INVALID_ARG;
+      if (hooks && hooks->before_stats_chunk) {
+        st = hooks->before_stats_chunk(t0, rows);
+        if (st != ULORL_OK) return st;
+      }
+      const int w_slabs = (c == 0 && hooks && hooks->before_w_slab) ? std::min(hooks->w_slabs, n_tiles) : 0;
+      if (w_slabs > 1) {
+        const int tiles_per_slab = (n_tiles + w_slabs - 1) / w_slabs;
+        const int s_loc = std::max(1, std::min(std::min(pl.n_split, pl.partial_slots / w_slabs), tiles_per_slab));
+        const int tps = (tiles_per_slab + s_loc - 1) / s_loc;
+        int k = 0;
+        for (int tile0 = 0; tile0 < n_tiles; tile0 += tiles_per_slab, ++k) {
+          const int tile1 = std::min(n_tiles, tile0 + tiles_per_slab);
+          const int v0 = tile0 * kBN, v1 = std::min(V, tile1 * kBN);
+          st = hooks->before_w_slab(k, v0, v1 - v0);
+          if (st != ULORL_OK) return st;
+          st = launch_stats(t0, rows, s_loc, tps, tile0, tile1, k * s_loc);
+          if (st != ULORL_OK) return st;
+        }
+        slab_tokens = rows;
+        slab_slots = k * s_loc;
+      } else {
+        st = launch_stats(t0, rows, pl.n_split, pl.tiles_per_split, 0, n_tiles, 0);
+        if (st != ULORL_OK) return st;
+      }
+    }
+    if (slab_tokens > 0) {
+      merge_splits_kernel<<<(slab_tokens + 255) / 256, 256, 0, stream>>>(T, 0, slab_tokens, slab_slots, kappa, partials,
+                                                                          acc_y, logp, entropy, lse);
+      ULORL_LAUNCH_CHECK();
+    }
+    if (slab_tokens < T) {
+      merge_splits_kernel<<<(T - slab_tokens + 255) / 256, 256, 0, stream>>>(T, slab_tokens, T, pl.n_split, kappa,
+                                                                              partials, acc_y, logp, entropy, lse);
+      ULORL_LAUNCH_CHECK();
     }
   } else {
     if (hooks && hooks->before_stats_chunk) {
@@ -547,9 +594,10 @@ static int fwd_impl(const ulorl_params_t* params, const void* hidden, const void
           static_cast<const __nv_bfloat16*>(hidden), static_cast<const __nv_bfloat16*>(W), targets, T, V, H, kappa,
           pl.tiles_per_split, partials, acc_y, status);
     ULORL_LAUNCH_CHECK();
+    merge_splits_kernel<<<(T + 255) / 256, 256, 0, stream>>>(T, 0, T, pl.n_split, kappa, partials, acc_y, logp, entropy,
+                                                             lse);
+    ULORL_LAUNCH_CHECK();
   }
-  merge_splits_kernel<<<(T + 255) / 256, 256, 0, stream>>>(T, pl.n_split, kappa, partials, acc_y, logp, entropy, lse);
-  ULORL_LAUNCH_CHECK();
   return run_decide(params, pl, logp, entropy, old_logp, segment_version, advantages, seq_offsets, entropy_supplied,
                     grad_coef, flags, seq_entropy, loss, stats, ws, stream);
 }
@@ -1073,25 +1121,66 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
   if (!ok(h2d(L.targets, h_targets, T * 4)) || !ok(h2d(L.old_logp, h_old_logp, T * 4)) ||
       !ok(h2d(L.segver, h_segment_version, T * 4)) ||
       !ok(h2d(L.adv, h_advantages, (params->adv_per_token ? T : S) * 4)) ||
-      !ok(h2d(L.seq_off, h_seq_offsets, (S + 1) * 4)) || !ok(h2d(L.ent_sup, h_entropy_supplied, S * 4)) ||
-      !ok(h2d(L.W, h_W, V * H * L.elem)))
+      !ok(h2d(L.seq_off, h_seq_offsets, (S + 1) * 4)) || !ok(h2d(L.ent_sup, h_entropy_supplied, S * 4)))
     return ULORL_ERR_CUDA;
-  // hidden states chunk by chunk, one event per chunk: the statistics kernel of a chunk starts as soon as
-  // its rows have landed while the later chunks are still on the bus
+  // Order on the inbound stream: the first chunk of hidden states, then W in slabs of vocabulary rows, then
+  // the other chunks, one event each.  The statistics kernel sweeps the first chunk slab by slab as W lands
+  // (tensor path), and every later chunk as soon as its rows are there, while the rest is still on the bus.
+  // The first chunk is sized so that one of its slab sweeps takes about as long as a slab's copy.
   const int chunk = pl.panel_tokens;
-  const int n_chunks = params->T > 0 ? (params->T + chunk - 1) / chunk : 0;
-  if (!hs->reserve((size_t)n_chunks)) return ULORL_ERR_CUDA;
-  for (int c = 0; c < n_chunks; ++c) {
-    const size_t t0 = (size_t)c * chunk, rows = (T - t0) < (size_t)chunk ? (T - t0) : (size_t)chunk;
-    if (!ok(h2d(L.hidden + t0 * row_bytes, static_cast<const uint8_t*>(h_hidden) + t0 * row_bytes, rows * row_bytes)) ||
-        !ok(cudaEventRecord(hs->chunk_in[c], hs->in)))
-      return ULORL_ERR_CUDA;
-  }
+  const int tile_m = pl.tensor ? kBM * pl.cta : kBM;
   StepHooks hooks;
-  hooks.chunk_tokens = chunk;
-  hooks.before_stats_chunk = [&](int t0, int rows) {   // the last chunk that [t0, t0 + rows) touches has landed
-    return ok(cudaStreamWaitEvent(stream, hs->chunk_in[(t0 + rows - 1) / chunk], 0)) ? ULORL_OK : ULORL_ERR_CUDA;
+  if (params->T > 0) {
+    int first = (int)align_up((size_t)chunk * 11 / 8, (size_t)tile_m);
+    if (first >= params->T) first = params->T;
+    hooks.chunk_starts.push_back(0);
+    for (int t0 = first; t0 < params->T; t0 += chunk) hooks.chunk_starts.push_back(t0);
+  }
+  const int n_chunks = (int)hooks.chunk_starts.size();
+  constexpr int kWSlabs = 8;
+  const int n_tiles_v = (params->V + kBN - 1) / kBN;
+  const int w_slabs = pl.tensor ? std::min(kWSlabs, std::min(n_tiles_v, pl.partial_slots)) : 1;
+  const size_t n_panels = params->T > 0 ? ((size_t)params->T + chunk - 1) / chunk : 0;   // events of the backward's panels
+  if (!hs->reserve(std::max((size_t)std::max(n_chunks, 1) + (size_t)w_slabs, n_panels))) return ULORL_ERR_CUDA;
+  auto chunk_rows = [&](int c) {
+    const size_t t0 = (size_t)hooks.chunk_starts[c];
+    const size_t t1 = c + 1 < n_chunks ? (size_t)hooks.chunk_starts[c + 1] : T;
+    return std::make_pair(t0, t1 - t0);
   };
+  auto send_chunk = [&](int c) {
+    const auto [t0, rows] = chunk_rows(c);
+    return ok(h2d(L.hidden + t0 * row_bytes, static_cast<const uint8_t*>(h_hidden) + t0 * row_bytes, rows * row_bytes)) &&
+           ok(cudaEventRecord(hs->chunk_in[c], hs->in));
+  };
+  if (n_chunks > 0 && !send_chunk(0)) return ULORL_ERR_CUDA;
+  {
+    // W slab k = vocabulary tiles [k * tiles_per_slab, ...): the same ranges the forward sweeps the first chunk in;
+    // its event is kept behind the chunk events in the same table
+    const int tiles_per_slab = (n_tiles_v + w_slabs - 1) / w_slabs;
+    int k = 0;
+    for (int tile0 = 0; tile0 < n_tiles_v; tile0 += tiles_per_slab, ++k) {
+      const size_t v0 = (size_t)tile0 * kBN, v1 = std::min(V, (size_t)(tile0 + tiles_per_slab) * kBN);
+      if (!ok(h2d(L.W + v0 * row_bytes, static_cast<const uint8_t*>(h_W) + v0 * row_bytes, (v1 - v0) * row_bytes)) ||
+          !ok(cudaEventRecord(hs->chunk_in[(size_t)std::max(n_chunks, 1) + k], hs->in)))
+        return ULORL_ERR_CUDA;
+    }
+  }
+  for (int c = 1; c < n_chunks; ++c)
+    if (!send_chunk(c)) return ULORL_ERR_CUDA;
+  auto chunk_of = [&](int t) {       // index of the chunk that holds token t
+    int c = 0;
+    while (c + 1 < n_chunks && hooks.chunk_starts[c + 1] <= t) ++c;
+    return c;
+  };
+  hooks.before_stats_chunk = [&](int t0, int rows) {   // the last chunk that [t0, t0 + rows) touches has landed
+    return ok(cudaStreamWaitEvent(stream, hs->chunk_in[chunk_of(t0 + rows - 1)], 0)) ? ULORL_OK : ULORL_ERR_CUDA;
+  };
+  if (pl.tensor && w_slabs > 1) {
+    hooks.w_slabs = w_slabs;
+    hooks.before_w_slab = [&](int k, int, int) {
+      return ok(cudaStreamWaitEvent(stream, hs->chunk_in[(size_t)std::max(n_chunks, 1) + k], 0)) ? ULORL_OK : ULORL_ERR_CUDA;
+    };
+  }
   // d_hidden rows of a panel go back on the outbound stream while the next panel is computed
   hooks.after_dhidden_panel = [&](int t0, int rows) {
     if (!h_d_hidden) return (int)ULORL_OK;

@@ -69,6 +69,8 @@ struct UmmaArgs {
   int m_tiles, n_tiles;     // ceil(M / rows per unit), ceil(N / columns per unit)
   int n_split;              // kModeStats: vocabulary splits; a unit is (token tile, split)
   int tiles_per_split;
+  int tile_base;            // kModeStats: first vocabulary tile of this launch (its splits start there; n_tiles is the
+  int split_base;           // end tile) and the slot of its split 0 in `partials` -- a launch may cover a vocabulary range
   int group_m;              // other modes: token tiles per raster group (tiles of a group run m-fastest)
   int a_mn0, a_k0;          // coordinate offsets of operand A in its tensor map (MN index, K index)
   int b_mn0, b_k0;
@@ -303,7 +305,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         int m_tile, n_begin, n_end;
         if (kMode == kModeStats) {
           m_tile = unit / args.n_split;
-          n_begin = (unit % args.n_split) * args.tiles_per_split;
+          n_begin = args.tile_base + (unit % args.n_split) * args.tiles_per_split;
           n_end = min(args.n_tiles, n_begin + args.tiles_per_split);
         } else {
           unit_to_tile(unit, args, m_tile, n_begin);
@@ -407,7 +409,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       for (int unit = worker; unit < n_units; unit += n_workers) {
         int n_tiles_here = 1;
         if (kMode == kModeStats) {
-          const int n_begin = (unit % args.n_split) * args.tiles_per_split;
+          const int n_begin = args.tile_base + (unit % args.n_split) * args.tiles_per_split;
           n_tiles_here = min(args.n_tiles, n_begin + args.tiles_per_split) - n_begin;
         }
         for (int t = 0; t < n_tiles_here; ++t, ++acc_iter) {
@@ -465,7 +467,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       if (kMode == kModeStats) {
         m_tile = unit / args.n_split;
         split = unit % args.n_split;
-        n_begin = split * args.tiles_per_split;
+        n_begin = args.tile_base + split * args.tiles_per_split;
         n_end = min(args.n_tiles, n_begin + args.tiles_per_split);
       } else {
         unit_to_tile(unit, args, m_tile, n_begin);
@@ -620,7 +622,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       }
 
       if (kMode == kModeStats && row_ok)
-        args.partials[(size_t)split * args.T_total + grow] = make_float4(run_m, run_s, run_u, 0.f);
+        args.partials[(size_t)(args.split_base + split) * args.T_total + grow] = make_float4(run_m, run_s, run_u, 0.f);
     }
   }
 

@@ -132,12 +132,16 @@ def test_full_size_workload_against_sampled_oracle(name):
     dH_ref, _ = O.backward(h_rows[sel], W_host, y_rows[sel], g_or[sel], op.inv_temperature, want_dW=False)
     dH_gpu = dH[torch.from_numpy(active).to(DEV)].float().cpu().numpy()
     assert rel_l2(dH_gpu, dH_ref) <= TOL_GRAD
-    # row by row: no row is off by more than the tolerance times a typical row norm.  (A row whose
-    # target probability is within 1e-5 of one has a gradient ~(1 - p) that float32 cannot resolve
-    # relative to itself; its absolute size is then far below the typical row's.)
+    # row by row.  dHidden[t] = kappa g_t ((1 - p_y) W_y - sum_{v != y} p_v W_v): a float32 error d in the row's
+    # log-prob moves the first term by kappa |g_t| p_y d |W_y| whatever the size of 1 - p_y, so a row whose target
+    # probability is close to one carries an absolute error that its own (tiny) norm cannot absorb.  With float32
+    # accumulation over H = 2048 and logits up to ~40 that d is a few 1e-5 (the forward's contract allows 2e-3);
+    # the bound takes 1e-4.
     row_err = np.linalg.norm(dH_gpu - dH_ref, axis=1)
     row_ref = np.linalg.norm(dH_ref, axis=1)
-    assert (row_err <= 3 * TOL_GRAD * np.maximum(row_ref, np.median(row_ref))).all()
+    w_y = np.linalg.norm(W_host[y_rows[sel]].astype(np.float64), axis=1)
+    floor = op.inv_temperature * np.abs(g_or[sel]) * 1e-4 * w_y
+    assert (row_err <= 3 * TOL_GRAD * row_ref + floor).all()
     inactive = rows[g[rows] == 0]
     if inactive.size:
         assert float(dH[torch.from_numpy(inactive).to(DEV)].float().abs().max()) == 0.0
