@@ -176,7 +176,9 @@ int ulorl_token_loss_decide(const ulorl_params_t* params,
  * first call outside any stream capture.  All calls on a device share the one array, which keeps
  * the previous call's contents (the call clears the status word itself): two calls whose kernels
  * can overlap on the GPU -- different streams without an ordering between them -- race on it and
- * give wrong results.  Calls on one stream are ordered and safe.
+ * give wrong results.  Calls on one stream are ordered and safe.  Device-side findings (sequence
+ * offsets out of order, clamped) land in the array's own status word: read it with
+ * ulorl_check_status(NULL, stream), or from stats->device_status.
  */
 #define ULORL_STATIC_MAX_TOKENS (1 << 20)
 #define ULORL_STATIC_MAX_SEQS   (1 << 16)
@@ -257,12 +259,30 @@ int ulorl_token_loss_bwd_slabs(const ulorl_params_t* params,
                                void* d_hidden, void* d_W, ulorl_dw_slab_fn on_slab, void* user,
                                void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* Synchronises the stream, reads the workspace status word and returns it: ULORL_OK, or
+/*
+ * The float32 thresholds the decision stage compares against for these params (pure host function):
+ * out[0] = ln tau (Eq. 9 read as logp >= ln tau), out[1] = ln(1 + clip_eps_high), out[2] = ln(1 - clip_eps_low)
+ * (the clip bounds of Eq. 7 / Eq. 10 on the log-ratio; -inf when clip_eps_low = 1).  Each is the float64
+ * logarithm of the float32 parameter rounded to float32, so that no transcendental sits in a comparison.
+ */
+int ulorl_decision_thresholds(const ulorl_params_t* params, float* out);
+
+/* Synchronises the stream, reads the workspace status word (workspace = NULL: the status word of the built-in
+ * scratch of ulorl_token_loss_decide_static on the current device) and returns it: ULORL_OK, or
  * ULORL_ERR_DEVICE_TIMEOUT, ULORL_ERR_INVALID_ARG (seq_offsets on the device were not
  * 0 = o[0] <= ... <= o[S] = T; the offending ranges were clamped), ULORL_ERR_BAD_TARGET, ULORL_ERR_CUDA. */
 int ulorl_check_status(void* workspace, void* cuda_stream);
 
 const char* ulorl_status_string(int status);
+
+/*
+ * Self-test of the failure path: launches one small block that waits, with the bounded wait the tensor-core
+ * kernels use, on a barrier nobody signals; after limit_cycles SM clocks (1e3 .. 1e8) the wait gives up, the
+ * block sets the timeout bit in the workspace status word and returns normally.  ulorl_check_status then
+ * reports ULORL_ERR_DEVICE_TIMEOUT; the next forward call clears the word.  Nothing else runs in the block:
+ * no copy, no tensor memory, so the context stays usable.
+ */
+int ulorl_selftest_bounded_wait(void* workspace, int64_t limit_cycles, void* cuda_stream);
 
 /* Number of kernel launches issued by this library since it was loaded (host counter). */
 int64_t ulorl_launch_count(void);

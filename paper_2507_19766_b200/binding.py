@@ -66,7 +66,7 @@ EXPORTS = ("ulorl_workspace_bytes", "ulorl_token_loss_fwd", "ulorl_token_loss_de
            "ulorl_check_status", "ulorl_status_string", "ulorl_launch_count", "ulorl_kernel_timing_begin",
            "ulorl_kernel_timing_end", "ulorl_host_step_arena_bytes", "ulorl_token_loss_step_host",
            "ulorl_token_loss_decide_static", "ulorl_group_advantages", "ulorl_sequence_entropy_partials",
-           "ulorl_sequence_entropy_combine")
+           "ulorl_sequence_entropy_combine", "ulorl_decision_thresholds", "ulorl_selftest_bounded_wait")
 STATIC_MAX_TOKENS, STATIC_MAX_SEQS = 1 << 20, 1 << 16
 KERNEL_KINDS = ("stats", "dz", "d_hidden", "d_W")
 
@@ -99,6 +99,10 @@ def load_library() -> ctypes.CDLL:
     lib.ulorl_sequence_entropy_partials.argtypes = [cp, vp, vp, vp, ctypes.c_int32, vp, vp, vp]
     lib.ulorl_sequence_entropy_combine.restype = ctypes.c_int
     lib.ulorl_sequence_entropy_combine.argtypes = [vp, ctypes.c_int32, vp, ctypes.c_int32, vp, vp, vp]
+    lib.ulorl_selftest_bounded_wait.restype = ctypes.c_int
+    lib.ulorl_selftest_bounded_wait.argtypes = [vp, ctypes.c_int64, vp]
+    lib.ulorl_decision_thresholds.restype = ctypes.c_int
+    lib.ulorl_decision_thresholds.argtypes = [cp, ctypes.POINTER(ctypes.c_float)]
     lib.ulorl_token_loss_bwd.restype = ctypes.c_int
     lib.ulorl_token_loss_bwd.argtypes = [cp] + [vp] * 8 + [vp, ctypes.c_size_t, vp]
     lib.ulorl_token_loss_bwd_slabs.restype = ctypes.c_int
@@ -175,6 +179,13 @@ def workspace_bytes(p: Params) -> int:
     if n == 0:
         raise UlorlError("ulorl_workspace_bytes: invalid parameters")
     return int(n)
+
+
+def decision_thresholds(p: Params):
+    """(ln tau, ln(1 + eps_high), ln(1 - eps_low)) as the float32 values the decision kernel compares with."""
+    out = (ctypes.c_float * 3)()
+    _check(load_library().ulorl_decision_thresholds(ctypes.byref(p.to_c()), out), "ulorl_decision_thresholds", "ulorl_selftest_bounded_wait")
+    return tuple(float(x) for x in out)
 
 
 def launch_count() -> int:
@@ -333,8 +344,14 @@ def token_loss_bwd(p: Params, hidden, W, targets, lse, grad_coef, grad_loss=None
     return d_hidden, d_W
 
 
-def check_status(workspace: torch.Tensor) -> int:
+def check_status(workspace: Optional[torch.Tensor]) -> int:
+    """ulorl_check_status; workspace=None reads the status word of the no-allocation entry point's built-in scratch."""
     return int(load_library().ulorl_check_status(_ptr(workspace), _stream()))
+
+
+def selftest_bounded_wait(workspace: torch.Tensor, limit_cycles: int = 1_000_000) -> int:
+    """ulorl_selftest_bounded_wait: returns the launch status; the timeout shows up in check_status(workspace)."""
+    return int(load_library().ulorl_selftest_bounded_wait(_ptr(workspace), limit_cycles, _stream()))
 
 
 def kernel_timing_begin():

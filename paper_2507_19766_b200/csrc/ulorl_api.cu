@@ -25,7 +25,6 @@ constexpr int kMaxDevices = 64;            // per-device set-up tables
 constexpr int kFallbackSMs = 148;         // B200; used for the plan when no device can be asked
 constexpr int kDefaultPanelTensor = 16384;       // single-CTA kernels
 constexpr int kDefaultPanelSimt = 1024;
-constexpr int kFirstChunkSlots = 16;      // partial slots a first chunk may use when W arrives in slabs (host-buffer step)
 constexpr int kRasterGroup = 16;          // dz: row tiles per raster group (m fastest inside a group)
 constexpr int kGradRasterGroup = 1;       // d_hidden, d_W: column blocks of one row tile run side by side, so its A stream is read once
 
@@ -60,7 +59,6 @@ struct Plan {
   int cta;                // CTAs per tcgen05.mma: 2 (a CTA pair per 256 x 256 tile) or 1 (ULORL_PATH_TENSOR_1CTA)
   int sms;                // multiprocessors the persistent kernels are spread over
   int n_split, tiles_per_split;
-  int partial_slots;      // slots per token in the softmax partials: n_split, or more for a first chunk swept slab by slab
   int panel_tokens;
   size_t dz_ld;           // leading dimension of the dz panel (elements)
   size_t off_status, off_batch_mean, off_seq_sum, off_partials, off_acc_y, off_decide, off_dz, total;
@@ -159,8 +157,7 @@ static Plan make_plan(const ulorl_params_t* p) {
   pl.off_status = off;      off += 256;
   pl.off_batch_mean = pl.off_status + 16;
   pl.off_seq_sum = off;     off = align_up(off + sizeof(long long) * (size_t)(p->num_seqs > 0 ? p->num_seqs : 1), 256);
-  pl.partial_slots = pl.tensor ? std::max(pl.n_split, std::min(kFirstChunkSlots, n_tiles)) : pl.n_split;
-  pl.off_partials = off;    off = align_up(off + sizeof(float4) * (size_t)pl.partial_slots * (size_t)(T > 0 ? T : 1), 256);
+  pl.off_partials = off;    off = align_up(off + sizeof(float4) * (size_t)pl.n_split * (size_t)(T > 0 ? T : 1), 256);
   pl.off_acc_y = off;       off = align_up(off + sizeof(float) * (size_t)(T > 0 ? T : 1), 256);
   pl.off_decide = off;      off = align_up(off + sizeof(DecidePartial) * (size_t)(pl.decide_blocks > 0 ? pl.decide_blocks : 1), 1024);
   pl.off_dz = off;          off = align_up(off + (size_t)panel * pl.dz_ld * (pl.tensor ? 2 : 4), 1024);
@@ -409,17 +406,23 @@ static int empty_forward(void* workspace, size_t workspace_bytes, float* loss, v
   return ULORL_OK;
 }
 
+// Vocabulary tiles of each split that one of `w_slabs` cuts of a sweep covers.
+static int w_slab_tiles(const Plan& pl, int w_slabs) {
+  return std::max(1, (pl.tiles_per_split + w_slabs - 1) / std::max(w_slabs, 1));
+}
+
 // Points at which the host-buffer step interleaves its copies with the two passes.  The forward
 // launches the statistics kernel once per chunk of tokens (all at once without hooks), the backward
 // reports every token panel whose d_hidden rows are final.
 struct StepHooks {
   // Forward, tensor path: the statistics kernel is launched once per chunk of tokens; chunk c covers tokens
   // [chunk_starts[c], chunk_starts[c + 1]) (the last one runs to T; empty = one chunk).  With w_slabs > 1 the
-  // FIRST chunk is swept in w_slabs launches, one per range of vocabulary tiles, and before_w_slab(k, first row,
-  // rows) is called before launch k: W may still be arriving while the chunk's first launches run.
+  // sweep of the FIRST chunk is cut into w_slabs launches: launch j covers, of every vocabulary split, the j-th
+  // run of tiles (w_slab_tiles(plan) of them), and before_w_slab(j) is called before it -- W may still be
+  // arriving while the chunk's first launches run.  The cut does not change the results.
   std::vector<int> chunk_starts;
   int w_slabs = 0;
-  std::function<int(int, int, int)> before_w_slab;
+  std::function<int(int)> before_w_slab;
   std::function<int(int, int)> before_stats_chunk;    // (first token, tokens) -> status
   std::function<int(int, int)> after_dhidden_panel;   // (first token, tokens) -> status; dense backward only
   // Tensor path: when set, the last panel computes d_W before d_hidden and in slabs of vocabulary rows,
@@ -438,6 +441,25 @@ size_t ulorl_workspace_bytes(const ulorl_params_t* params) {
   return make_plan(params).total;
 }
 
+int ulorl_selftest_bounded_wait(void* workspace, int64_t limit_cycles, void* cuda_stream) {
+  if (!workspace) return ULORL_ERR_INVALID_ARG;
+  if (limit_cycles < 1000 || limit_cycles > 100000000) return ULORL_ERR_INVALID_ARG;   // at most ~0.1 s of SM clocks
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  bounded_wait_selftest_kernel<<<1, 32, 0, stream>>>((long long)limit_cycles, reinterpret_cast<int*>(workspace));
+  return check_launch();
+}
+
+int ulorl_decision_thresholds(const ulorl_params_t* params, float* out) {
+  const int st = validate_params(params);
+  if (st != ULORL_OK) return st;
+  if (!out) return ULORL_ERR_INVALID_ARG;
+  const DecideConsts c = make_decide_consts(params);
+  out[0] = c.ln_tau;
+  out[1] = c.ln_hi;
+  out[2] = c.ln_lo;
+  return ULORL_OK;
+}
+
 int64_t ulorl_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
 
 const char* ulorl_status_string(int status) {
@@ -454,8 +476,15 @@ const char* ulorl_status_string(int status) {
   }
 }
 
+static int static_scratch_address(uint8_t** out);
+
 int ulorl_check_status(void* workspace, void* cuda_stream) {
-  if (!workspace) return ULORL_ERR_INVALID_ARG;
+  if (!workspace) {   // the status word of the built-in scratch of ulorl_token_loss_decide_static on this device
+    uint8_t* builtin = nullptr;
+    const int st = static_scratch_address(&builtin);
+    if (st != ULORL_OK) return st;
+    workspace = builtin;
+  }
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   int word = 0;
   if (cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return ULORL_ERR_CUDA;
@@ -519,16 +548,16 @@ static int fwd_impl(const ulorl_params_t* params, const void* hidden, const void
     const int n_tiles = (V + kBN - 1) / kBN;
     std::vector<int> starts = (hooks && !hooks->chunk_starts.empty()) ? hooks->chunk_starts : std::vector<int>{0};
     starts.push_back(T);
-    auto launch_stats = [&](int t0, int rows, int n_split, int tiles_per_split, int tile_base, int tile_end,
-                            int split_base) -> int {
+    auto launch_stats = [&](int t0, int rows, int tile_base, int tiles, int resume) -> int {
       UmmaArgs a{};
       a.M = rows; a.N = V; a.K = H;
       a.m_tiles = (rows + tile_m - 1) / tile_m;
-      a.n_tiles = tile_end;
-      a.n_split = n_split;
-      a.tiles_per_split = tiles_per_split;
+      a.n_tiles = n_tiles;
+      a.n_split = pl.n_split;
+      a.split_stride = pl.tiles_per_split;
+      a.tiles_per_split = tiles;
       a.tile_base = tile_base;
-      a.split_base = split_base;
+      a.resume = resume;
       a.a_mn0 = t0;
       a.row0 = t0;
       a.kappa = kappa;
@@ -539,8 +568,6 @@ static int fwd_impl(const ulorl_params_t* params, const void* hidden, const void
       a.status = status;
       return launch_umma<kModeStats>(pl, map_a, map_b, map_a, a, stream);
     };
-    // tokens [0, slab_rows_end) get their statistics from w_slabs launches over vocabulary ranges
-    int slab_tokens = 0, slab_slots = 0;
     for (size_t c = 0; c + 1 < starts.size(); ++c) {
       const int t0 = starts[c], rows = starts[c + 1] - starts[c];
       if (rows <= 0 || t0 % tile_m != 0) return ULORL_ERR_INVALID_ARG;
@@ -548,37 +575,23 @@ static int fwd_impl(const ulorl_params_t* params, const void* hidden, const void
         st = hooks->before_stats_chunk(t0, rows);
         if (st != ULORL_OK) return st;
       }
-      const int w_slabs = (c == 0 && hooks && hooks->before_w_slab) ? std::min(hooks->w_slabs, n_tiles) : 0;
+      const int w_slabs = (c == 0 && hooks && hooks->before_w_slab) ? hooks->w_slabs : 0;
       if (w_slabs > 1) {
-        const int tiles_per_slab = (n_tiles + w_slabs - 1) / w_slabs;
-        const int s_loc = std::max(1, std::min(std::min(pl.n_split, pl.partial_slots / w_slabs), tiles_per_slab));
-        const int tps = (tiles_per_slab + s_loc - 1) / s_loc;
-        int k = 0;
-        for (int tile0 = 0; tile0 < n_tiles; tile0 += tiles_per_slab, ++k) {
-          const int tile1 = std::min(n_tiles, tile0 + tiles_per_slab);
-          const int v0 = tile0 * kBN, v1 = std::min(V, tile1 * kBN);
-          st = hooks->before_w_slab(k, v0, v1 - v0);
+        const int q = w_slab_tiles(pl, w_slabs);
+        for (int j = 0; j * q < pl.tiles_per_split; ++j) {
+          st = hooks->before_w_slab(j);
           if (st != ULORL_OK) return st;
-          st = launch_stats(t0, rows, s_loc, tps, tile0, tile1, k * s_loc);
+          st = launch_stats(t0, rows, j * q, q, j > 0 ? 1 : 0);
           if (st != ULORL_OK) return st;
         }
-        slab_tokens = rows;
-        slab_slots = k * s_loc;
       } else {
-        st = launch_stats(t0, rows, pl.n_split, pl.tiles_per_split, 0, n_tiles, 0);
+        st = launch_stats(t0, rows, 0, pl.tiles_per_split, 0);
         if (st != ULORL_OK) return st;
       }
     }
-    if (slab_tokens > 0) {
-      merge_splits_kernel<<<(slab_tokens + 255) / 256, 256, 0, stream>>>(T, 0, slab_tokens, slab_slots, kappa, partials,
-                                                                          acc_y, logp, entropy, lse);
-      ULORL_LAUNCH_CHECK();
-    }
-    if (slab_tokens < T) {
-      merge_splits_kernel<<<(T - slab_tokens + 255) / 256, 256, 0, stream>>>(T, slab_tokens, T, pl.n_split, kappa,
-                                                                              partials, acc_y, logp, entropy, lse);
-      ULORL_LAUNCH_CHECK();
-    }
+    merge_splits_kernel<<<(T + 255) / 256, 256, 0, stream>>>(T, 0, T, pl.n_split, kappa, partials, acc_y, logp, entropy,
+                                                             lse);
+    ULORL_LAUNCH_CHECK();
   } else {
     if (hooks && hooks->before_stats_chunk) {
       st = hooks->before_stats_chunk(0, T);
@@ -1139,9 +1152,10 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
   const int n_chunks = (int)hooks.chunk_starts.size();
   constexpr int kWSlabs = 8;
   const int n_tiles_v = (params->V + kBN - 1) / kBN;
-  const int w_slabs = pl.tensor ? std::min(kWSlabs, std::min(n_tiles_v, pl.partial_slots)) : 1;
+  const int w_slabs = pl.tensor ? std::max(1, std::min(kWSlabs, pl.tiles_per_split)) : 1;
   const size_t n_panels = params->T > 0 ? ((size_t)params->T + chunk - 1) / chunk : 0;   // events of the backward's panels
   if (!hs->reserve(std::max((size_t)std::max(n_chunks, 1) + (size_t)w_slabs, n_panels))) return ULORL_ERR_CUDA;
+  const size_t w_event0 = (size_t)std::max(n_chunks, 1);   // W-slab events sit behind the chunk events in the same table
   auto chunk_rows = [&](int c) {
     const size_t t0 = (size_t)hooks.chunk_starts[c];
     const size_t t1 = c + 1 < n_chunks ? (size_t)hooks.chunk_starts[c + 1] : T;
@@ -1154,15 +1168,21 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
   };
   if (n_chunks > 0 && !send_chunk(0)) return ULORL_ERR_CUDA;
   {
-    // W slab k = vocabulary tiles [k * tiles_per_slab, ...): the same ranges the forward sweeps the first chunk in;
-    // its event is kept behind the chunk events in the same table
-    const int tiles_per_slab = (n_tiles_v + w_slabs - 1) / w_slabs;
-    int k = 0;
-    for (int tile0 = 0; tile0 < n_tiles_v; tile0 += tiles_per_slab, ++k) {
-      const size_t v0 = (size_t)tile0 * kBN, v1 = std::min(V, (size_t)(tile0 + tiles_per_slab) * kBN);
-      if (!ok(h2d(L.W + v0 * row_bytes, static_cast<const uint8_t*>(h_W) + v0 * row_bytes, (v1 - v0) * row_bytes)) ||
-          !ok(cudaEventRecord(hs->chunk_in[(size_t)std::max(n_chunks, 1) + k], hs->in)))
-        return ULORL_ERR_CUDA;
+    // W slab j = of every vocabulary split of the statistics kernel, its j-th run of tiles: exactly what cut j
+    // of the first chunk's sweep reads
+    const int q = pl.tensor ? w_slab_tiles(pl, w_slabs) : n_tiles_v;
+    const int stride = pl.tensor ? pl.tiles_per_split : n_tiles_v;
+    const int splits = pl.tensor ? pl.n_split : 1;
+    for (int j = 0; j * q < stride; ++j) {
+      for (int sp = 0; sp < splits; ++sp) {
+        const int tile0 = sp * stride + j * q;
+        const int tile1 = std::min(std::min(tile0 + q, (sp + 1) * stride), n_tiles_v);
+        if (tile1 <= tile0) continue;
+        const size_t v0 = (size_t)tile0 * kBN, v1 = std::min(V, (size_t)tile1 * kBN);
+        if (!ok(h2d(L.W + v0 * row_bytes, static_cast<const uint8_t*>(h_W) + v0 * row_bytes, (v1 - v0) * row_bytes)))
+          return ULORL_ERR_CUDA;
+      }
+      if (j < w_slabs && !ok(cudaEventRecord(hs->chunk_in[w_event0 + j], hs->in))) return ULORL_ERR_CUDA;
     }
   }
   for (int c = 1; c < n_chunks; ++c)
@@ -1177,8 +1197,8 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
   };
   if (pl.tensor && w_slabs > 1) {
     hooks.w_slabs = w_slabs;
-    hooks.before_w_slab = [&](int k, int, int) {
-      return ok(cudaStreamWaitEvent(stream, hs->chunk_in[(size_t)std::max(n_chunks, 1) + k], 0)) ? ULORL_OK : ULORL_ERR_CUDA;
+    hooks.before_w_slab = [&](int j) {
+      return ok(cudaStreamWaitEvent(stream, hs->chunk_in[w_event0 + j], 0)) ? ULORL_OK : ULORL_ERR_CUDA;
     };
   }
   // d_hidden rows of a panel go back on the outbound stream while the next panel is computed

@@ -69,8 +69,12 @@ struct UmmaArgs {
   int m_tiles, n_tiles;     // ceil(M / rows per unit), ceil(N / columns per unit)
   int n_split;              // kModeStats: vocabulary splits; a unit is (token tile, split)
   int tiles_per_split;
-  int tile_base;            // kModeStats: first vocabulary tile of this launch (its splits start there; n_tiles is the
-  int split_base;           // end tile) and the slot of its split 0 in `partials` -- a launch may cover a vocabulary range
+  // kModeStats: split s owns the vocabulary tiles [s * split_stride, (s + 1) * split_stride); a launch sweeps the
+  // tiles_per_split tiles of each split that start at offset tile_base inside it.  A whole sweep has tile_base = 0
+  // and tiles_per_split = split_stride; a sweep cut into several launches (W still arriving) sets `resume` on
+  // all but the first, and a row's running (max, sum, sum) then continues from `partials` exactly where the
+  // launch before left it, so the cut does not change a bit of the result.
+  int split_stride, tile_base, resume;
   int group_m;              // other modes: token tiles per raster group (tiles of a group run m-fastest)
   int a_mn0, a_k0;          // coordinate offsets of operand A in its tensor map (MN index, K index)
   int b_mn0, b_k0;
@@ -112,6 +116,14 @@ __device__ __forceinline__ void unit_to_tile(int unit, const UmmaArgs& args, int
   const int local = unit - group * per_group;
   m_tile = first_m + local % rows;
   n_tile = local / rows;
+}
+
+// Vocabulary tiles [n_begin, n_end) that this launch sweeps for split `split` (kModeStats); may be empty.
+__device__ __forceinline__ void stats_tile_range(const UmmaArgs& args, int split, int& n_begin, int& n_end) {
+  const int first = split * args.split_stride;
+  n_begin = first + args.tile_base;
+  n_end = min(min(n_begin + args.tiles_per_split, first + args.split_stride), args.n_tiles);
+  if (n_end < n_begin) n_end = n_begin;
 }
 
 __device__ __forceinline__ float ex2f(float x) {
@@ -305,8 +317,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         int m_tile, n_begin, n_end;
         if (kMode == kModeStats) {
           m_tile = unit / args.n_split;
-          n_begin = args.tile_base + (unit % args.n_split) * args.tiles_per_split;
-          n_end = min(args.n_tiles, n_begin + args.tiles_per_split);
+          stats_tile_range(args, unit % args.n_split, n_begin, n_end);
         } else {
           unit_to_tile(unit, args, m_tile, n_begin);
           n_end = n_begin + 1;
@@ -409,8 +420,9 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       for (int unit = worker; unit < n_units; unit += n_workers) {
         int n_tiles_here = 1;
         if (kMode == kModeStats) {
-          const int n_begin = args.tile_base + (unit % args.n_split) * args.tiles_per_split;
-          n_tiles_here = min(args.n_tiles, n_begin + args.tiles_per_split) - n_begin;
+          int n_begin, n_end;
+          stats_tile_range(args, unit % args.n_split, n_begin, n_end);
+          n_tiles_here = n_end - n_begin;
         }
         for (int t = 0; t < n_tiles_here; ++t, ++acc_iter) {
           const uint32_t buf = acc_iter % kBufs;
@@ -467,8 +479,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       if (kMode == kModeStats) {
         m_tile = unit / args.n_split;
         split = unit % args.n_split;
-        n_begin = args.tile_base + split * args.tiles_per_split;
-        n_end = min(args.n_tiles, n_begin + args.tiles_per_split);
+        stats_tile_range(args, split, n_begin, n_end);
       } else {
         unit_to_tile(unit, args, m_tile, n_begin);
         n_end = n_begin + 1;
@@ -489,6 +500,10 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             y = y < 0 ? 0 : args.N - 1;
           }
         }
+      }
+      if (kMode == kModeStats && args.resume && row_ok) {  // continue the sweep the launch before left off
+        const float4 p = args.partials[(size_t)split * args.T_total + grow];
+        run_m = p.x; run_s = p.y; run_u = p.z;
       }
       float k_row = -INFINITY;                          // kModeDz: log2|coef| - lse log2(e); -inf gives a zero row
       uint32_t sign_mask = 0u;
@@ -622,7 +637,7 @@ umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       }
 
       if (kMode == kModeStats && row_ok)
-        args.partials[(size_t)(args.split_base + split) * args.T_total + grow] = make_float4(run_m, run_s, run_u, 0.f);
+        args.partials[(size_t)split * args.T_total + grow] = make_float4(run_m, run_s, run_u, 0.f);
     }
   }
 
@@ -636,6 +651,25 @@ role_done:
     tc_fence_after_sync();
     if (kPair) tmem_dealloc_pair(tmem_base, kTmemCols);
     else tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// The bounded wait on its own: one block, one mbarrier on which nobody ever arrives, no copy and no tensor
+// memory in flight.  The wait gives up after limit_cycles, the kernel records the timeout in the status word
+// and returns normally -- the way umma_kernel reports a stall, exercised without stalling anything.
+__global__ void bounded_wait_selftest_kernel(long long limit_cycles, int* status) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    ptx::mbar_init(ptx::smem_u32(&bar), 1);
+    ptx::mbar_fence_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    volatile int* abort_p = &abort_flag;
+    const bool done = ptx::mbar_wait_bounded(ptx::smem_u32(&bar), 0u, abort_p, limit_cycles);
+    if (!done) atomicOr(status, kStatusTimeout);
   }
 }
 

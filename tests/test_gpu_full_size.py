@@ -147,9 +147,21 @@ def test_full_size_workload_against_sampled_oracle(name):
         assert float(dH[torch.from_numpy(inactive).to(DEV)].float().abs().max()) == 0.0
 
     # ---- dW: properties at full size
-    col = float(dW.double().sum(dim=0).abs().max())
+    # column sums of d_W vanish up to the bf16 rounding of dz: six standard deviations of independent roundings
+    # (2^-9 sqrt(2) |coef_t| per token) plus the float32 part that adds up linearly; the worst case behind it
+    colsum = dW.double().sum(dim=0).abs()
+    coef_t = out.grad_coef.abs().double() * op.inv_temperature
+    stat = torch.zeros(wl.H, dtype=torch.float64, device=DEV)
+    syst = torch.zeros(wl.H, dtype=torch.float64, device=DEV)
+    for a in range(0, wl.T, 16384):
+        ch = coef_t[a:a + 16384, None] * b.hidden[a:a + 16384].double().abs()
+        stat += (ch * ch).sum(dim=0)
+        syst += ch.sum(dim=0)
+    bound = 6.0 * 2.0 ** -9 * np.sqrt(2.0) * stat.sqrt() + 4e-6 * syst + 1e-12
+    assert bool((colsum <= bound).all()), float((colsum / bound).max())
     coef_sum = float(np.abs(g).sum()) * op.inv_temperature
-    assert col <= 2.0 ** -8 * coef_sum * float(batch.hidden.float().abs().max()) + 1e-12
+    assert float(colsum.max()) <= 2.0 ** -8 * coef_sum * float(batch.hidden.float().abs().max()) + 1e-12
+    print(f"{name}: d_W column sums at most {float((colsum / bound).max()):.3f} of the statistical bound")
     assert torch.isfinite(dW).all()
     dW_host = dW.cpu()
     del dW, dH

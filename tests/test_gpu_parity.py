@@ -14,6 +14,7 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 STAT_KEYS = ("n_tokens", "n_active", "n_mpt", "n_masked", "n_clip_high", "n_clip_low")
+COLSUM_MARGINS = []      # largest |column sum of d_W| / statistical bound seen by each parity case (reported at the end)
 
 
 def gpu_fwd_bwd(batch, gp, grad_loss=None, entropy_supplied=None):
@@ -102,13 +103,23 @@ def check_against_oracle(batch, gp, op, grad_loss=None, check_grads=True):
         eh = rel_l2(dH.float().cpu().numpy(), dH_ref)
         ew = rel_l2(dW.cpu().numpy(), dW_ref)
         assert eh <= TOL_GRAD and ew <= TOL_GRAD, (eh, ew)
-        # sum_v dz[t, v] = 0, so the column sums of d_W vanish up to the rounding of dz: the tensor path
-        # stores dz in bf16 (relative error 2^-9 per element, sum_v |dz[t, v]| <= 2 |coef_t|), so
-        # |colsum_h| <= 2^-8 sum_t |coef_t| |hidden[t, h]|; the float32 path is held to 1e-5 of that sum
-        col = np.abs(dW.double().sum(dim=0).cpu().numpy()).max()
-        coef_sum = float(np.abs(ref["grad_coef"]).sum()) * op.inv_temperature * abs(gl) * 1.01
-        unit = 2.0 ** -8 if (gp.dtype == "bf16" and gp.kernel_path != "simt") else 1e-5
-        assert col <= unit * coef_sum * float(np.abs(oi["hidden"]).max()) + 1e-12
+        # sum_v dz[t, v] = 0, so the column sums of d_W vanish up to the rounding of dz.  The tensor path stores dz in
+        # bf16: every element carries an independent relative error of at most 2^-9, so the error of sum_v dz[t, v]
+        # has a standard deviation below e_t = 2^-9 |dz_t|_2 <= 2^-9 sqrt(2) |coef_t|, and the column sum over T
+        # tokens one below sqrt(sum_t (e_t hidden[t, h])^2).  Held to six of those, plus the systematic part that
+        # does add up linearly: softmax rows that sum to one only to float32 (4e-6 sum_t |coef_t hidden[t, h]|).
+        # The float32 path has no bf16 step (1e-6 in place of 2^-9).  The worst-case bound (all roundings aligned)
+        # is kept behind it; it never binds.
+        colsum = np.abs(dW.double().sum(dim=0).cpu().numpy())
+        coef = np.abs(ref["grad_coef"]) * op.inv_temperature * abs(gl)
+        habs = np.abs(oi["hidden"]).astype(np.float64)
+        unit = 2.0 ** -9 * np.sqrt(2.0) if (gp.dtype == "bf16" and gp.kernel_path != "simt") else 1e-6
+        stat = 6.0 * unit * np.sqrt(((coef[:, None] * habs) ** 2).sum(axis=0))
+        syst = 4e-6 * (coef[:, None] * habs).sum(axis=0)
+        assert (colsum <= stat + syst + 1e-12).all(), float((colsum / (stat + syst + 1e-12)).max())
+        worst = 2.0 ** -8 if (gp.dtype == "bf16" and gp.kernel_path != "simt") else 1e-5
+        assert colsum.max() <= worst * float(coef.sum()) * 1.01 * float(habs.max()) + 1e-12
+        COLSUM_MARGINS.append(float((colsum / (stat + syst + 1e-12)).max()))
     return out, ref
 
 
@@ -720,3 +731,11 @@ def test_slab_wise_all_reduce_on_a_one_rank_nccl_group():
     finally:
         if created:
             dist.destroy_process_group()
+
+
+def test_zz_report_colsum_margins():
+    """Not a check of its own: prints how close the d_W column sums came to their statistical bound."""
+    if COLSUM_MARGINS:
+        print(f"d_W column sums: largest fraction of the statistical bound over {len(COLSUM_MARGINS)} cases = "
+              f"{max(COLSUM_MARGINS):.3f}")
+        assert max(COLSUM_MARGINS) <= 1.0

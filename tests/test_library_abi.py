@@ -68,3 +68,34 @@ def test_null_arguments_are_rejected_without_a_device(lib):
     code = lib.ulorl_token_loss_bwd(ctypes.byref(p), *([None] * 8), None, 0, None)
     assert code == -1
     assert lib.ulorl_token_loss_fwd(None, *args, None, 0, None) == -1
+
+
+def golden_thresholds():
+    rows = []
+    for line in open(os.path.join(ROOT, "tests", "golden", "decision_thresholds.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        kind, pbits, _, vbits, _ = line.split()
+        rows.append((kind, int(pbits, 16), int(vbits, 16)))
+    return rows
+
+
+def test_decision_thresholds_of_the_library_match_the_correctly_rounded_logarithms(lib):
+    """The bit-exact decision contract rests on these float32 constants; the golden values come from a
+    60-digit decimal logarithm (tests/golden/make_decision_thresholds.py), not from libm."""
+    import struct
+    f = lambda b: struct.unpack("<f", struct.pack("<I", b))[0]
+    bits = lambda x: struct.unpack("<I", struct.pack("<f", x))[0]
+    seen = set()
+    for kind, pbits, vbits in golden_thresholds():
+        kw = dict(T=8, H=64, V=128, num_seqs=1)
+        if kind == "ln_tau":
+            got = B.decision_thresholds(B.Params(mpt_tau=f(pbits), **kw))[0]
+        elif kind == "ln_1p_eps":
+            got = B.decision_thresholds(B.Params(clip_eps_high=f(pbits), **kw))[1]
+        else:
+            got = B.decision_thresholds(B.Params(clip_eps_low=f(pbits), **kw))[2]
+        assert bits(got) == vbits, (kind, hex(pbits), hex(bits(got)), hex(vbits))
+        seen.add(kind)
+    assert seen == {"ln_tau", "ln_1p_eps", "ln_1m_eps"}
+    assert B.decision_thresholds(B.Params(clip_eps_low=1.0, T=8, H=64, V=128, num_seqs=1))[2] == float("-inf")

@@ -342,6 +342,29 @@ def test_threshold_strictness():
         assert bool(out["flags"][0] & O.FLAG_CLIP_LOW) == expect
 
 
+def test_decision_thresholds_are_the_correctly_rounded_logarithms():
+    """decision_thresholds against float32 bit patterns from a 60-digit decimal logarithm of the exact float32
+    parameter (tests/golden/decision_thresholds.txt, written by make_decision_thresholds.py): the constants the
+    bit-exact mask and clip decisions rest on have a value that does not come from libm."""
+    seen = 0
+    path = os.path.join(os.path.dirname(__file__), "golden", "decision_thresholds.txt")
+    for line in open(path):
+        if line.startswith("#") or not line.strip():
+            continue
+        kind, pbits, _, vbits, _ = line.split()
+        param = float(np.array([int(pbits, 16)], dtype=np.uint32).view(np.float32)[0])
+        want = np.array([int(vbits, 16)], dtype=np.uint32).view(np.float32)[0]
+        if kind == "ln_tau":
+            got = O.decision_thresholds(O.OracleParams(mpt_tau=param))[0]
+        elif kind == "ln_1p_eps":
+            got = O.decision_thresholds(O.OracleParams(clip_eps_high=param))[1]
+        else:
+            got = O.decision_thresholds(O.OracleParams(clip_eps_low=param))[2]
+        assert got.dtype == np.float32 and got.view(np.uint32) == want.view(np.uint32), (kind, param, got, want)
+        seen += 1
+    assert seen == 9
+
+
 def test_entropy_scopes_and_sequence_means():
     ent = np.array([0.5, 1.5, 0.25, 0.75, 4.0], np.float32)
     offsets = np.array([0, 2, 4, 5])

@@ -54,6 +54,19 @@ def test_static_scratch_variant_matches_workspace_variant_twice_in_a_row():
         assert got.stats_host()["n_tokens"] == T and got.stats_host()["device_status"] == 0
 
 
+def test_static_scratch_variant_reports_bad_offsets_through_its_own_status_word():
+    # this caller has no workspace to ask: the finding is in the built-in array's status word
+    logp, ent, old, version, adv, offsets = make_case(33, 500, 3)
+    p = B.Params(T=500, H=8, V=16, num_seqs=3, dtype="f32", current_version=5)
+    out = B.alloc_fwd_outputs(p, DEV)
+    bad = offsets.clone()
+    bad[1] = 9999
+    B.token_loss_decide_static(p, logp, ent, old, version, adv, bad, out=out)
+    assert B.check_status(None) == -1 and out.stats_host()["device_status"] != 0
+    B.token_loss_decide_static(p, logp, ent, old, version, adv, offsets, out=out)
+    assert B.check_status(None) == B.OK and out.stats_host()["device_status"] == 0
+
+
 def test_static_scratch_variant_rejects_batches_beyond_its_limit():
     lib = B.load_library()
     for T, S in ((B.STATIC_MAX_TOKENS + 1, 1), (B.STATIC_MAX_SEQS + 1, B.STATIC_MAX_SEQS + 1)):
