@@ -184,7 +184,7 @@ def workspace_bytes(p: Params) -> int:
 def decision_thresholds(p: Params):
     """(ln tau, ln(1 + eps_high), ln(1 - eps_low)) as the float32 values the decision kernel compares with."""
     out = (ctypes.c_float * 3)()
-    _check(load_library().ulorl_decision_thresholds(ctypes.byref(p.to_c()), out), "ulorl_decision_thresholds", "ulorl_selftest_bounded_wait")
+    _check(load_library().ulorl_decision_thresholds(ctypes.byref(p.to_c()), out), "ulorl_decision_thresholds")
     return tuple(float(x) for x in out)
 
 

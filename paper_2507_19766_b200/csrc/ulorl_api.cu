@@ -1167,6 +1167,7 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
            ok(cudaEventRecord(hs->chunk_in[c], hs->in));
   };
   if (n_chunks > 0 && !send_chunk(0)) return ULORL_ERR_CUDA;
+  int n_w_events = 0;
   {
     // W slab j = of every vocabulary split of the statistics kernel, its j-th run of tiles: exactly what cut j
     // of the first chunk's sweep reads
@@ -1183,6 +1184,7 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
           return ULORL_ERR_CUDA;
       }
       if (j < w_slabs && !ok(cudaEventRecord(hs->chunk_in[w_event0 + j], hs->in))) return ULORL_ERR_CUDA;
+      n_w_events = std::min(j + 1, w_slabs);
     }
   }
   for (int c = 1; c < n_chunks; ++c)
@@ -1192,10 +1194,16 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
     while (c + 1 < n_chunks && hooks.chunk_starts[c + 1] <= t) ++c;
     return c;
   };
+  const bool sweep_by_slabs = pl.tensor && w_slabs > 1;
   hooks.before_stats_chunk = [&](int t0, int rows) {   // the last chunk that [t0, t0 + rows) touches has landed
-    return ok(cudaStreamWaitEvent(stream, hs->chunk_in[chunk_of(t0 + rows - 1)], 0)) ? ULORL_OK : ULORL_ERR_CUDA;
+    if (!ok(cudaStreamWaitEvent(stream, hs->chunk_in[chunk_of(t0 + rows - 1)], 0))) return (int)ULORL_ERR_CUDA;
+    // W follows the first chunk on the inbound stream: without the slab-wise sweep all of it must be there
+    if (!sweep_by_slabs && n_w_events > 0 &&
+        !ok(cudaStreamWaitEvent(stream, hs->chunk_in[w_event0 + n_w_events - 1], 0)))
+      return (int)ULORL_ERR_CUDA;
+    return (int)ULORL_OK;
   };
-  if (pl.tensor && w_slabs > 1) {
+  if (sweep_by_slabs) {
     hooks.w_slabs = w_slabs;
     hooks.before_w_slab = [&](int j) {
       return ok(cudaStreamWaitEvent(stream, hs->chunk_in[w_event0 + j], 0)) ? ULORL_OK : ULORL_ERR_CUDA;
