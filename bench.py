@@ -388,6 +388,37 @@ def e2e_run(leg: Leg, steps: int, dw_dtype: str) -> dict:
             "loss": float(ho["loss"][0])}
 
 
+def library_gemm_reference(ctx: Context, seconds: float = 4.0) -> dict:
+    """Context, not part of the path: the vendor library's bf16 GEMM (torch.matmul, 8192^3 and the LM-head shape
+    with the logits written out) run for a few seconds right behind the legs above, i.e. in the thermal and
+    power state they left.  Under the power cap the clock a kernel gets depends on that state, so this is the
+    like-for-like denominator for the legs that ran last."""
+    out = []
+    for M, N, K in ((8192, 8192, 8192), (16384, 16384, 2048)):
+        a = torch.randn(M, K, device=ctx.dev, dtype=torch.bfloat16)
+        b = torch.randn(N, K, device=ctx.dev, dtype=torch.bfloat16)
+        c = torch.empty(M, N, device=ctx.dev, dtype=torch.bfloat16)
+        for _ in range(3):
+            torch.matmul(a, b.t(), out=c)
+        torch.cuda.synchronize()
+        sampler = ClockSampler(ctx.local_rank).start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n, t0 = 0, time.perf_counter()
+        e0.record()
+        while time.perf_counter() - t0 < seconds / 2:
+            for _ in range(20):
+                torch.matmul(a, b.t(), out=c)
+            n += 20
+            torch.cuda.synchronize()
+        e1.record()
+        torch.cuda.synchronize()
+        clk = sampler.stop()
+        out.append({"kernel": "torch.matmul bf16 (cuBLAS)", "M": M, "N": N, "K": K,
+                    "tflops": 2.0 * M * N * K * n / (e0.elapsed_time(e1) * 1e-3) / 1e12, "clocks": clk})
+        del a, b, c
+    return {"note": "library GEMM in the state the last legs left the GPU in; context only", "runs": out}
+
+
 def run_ours(args, world, rank, local_rank):
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
@@ -474,6 +505,8 @@ def run_ours(args, world, rank, local_rank):
             del lo
             torch.cuda.empty_cache()
 
+    library_ref = library_gemm_reference(ctx) if full else None
+
     if rank != 0:
         if ctx.dist is not None:
             ctx.dist.destroy_process_group()
@@ -494,7 +527,7 @@ def run_ours(args, world, rank, local_rank):
         "loss": stats["loss"], "mean_entropy": stats["mean_entropy"], "n_masked": stats["n_masked"],
         "n_active": stats["n_active"],
         "roofline": roofline, "gate_shut": gate_shut, "other_workloads": others, "compacted": compacted,
-        "e2e": e2e, "e2e_bf16_dw": e2e_bf16, "comm": comm,
+        "e2e": e2e, "e2e_bf16_dw": e2e_bf16, "comm": comm, "library_gemm_same_state": library_ref,
         "gpu_launches": t_main["launches"], "clocks": main["clocks"],
     }
     if world == 1 and args.cpu_rows > 0:

@@ -164,8 +164,8 @@ int ulorl_token_loss_decide(const ulorl_params_t* params,
  * has no counterpart to this function; it is a packaging variant, not a step of the method.)
  *
  * The scratch that ulorl_token_loss_decide takes from the caller's workspace (status word,
- * per-sequence float64 entropy sums, one partial record per 256 tokens) lives instead in a fixed
- * array inside the library's device image: about 1.7 MB on every GPU that loads the library,
+ * per-sequence 64-bit entropy sums, one partial record per 1024 tokens) lives instead in a fixed
+ * array inside the library's device image: about 0.8 MB on every GPU that loads the library,
  * held until the process exits.  Limits: T <= ULORL_STATIC_MAX_TOKENS and num_seqs <=
  * ULORL_STATIC_MAX_SEQS; larger batches are rejected with ULORL_ERR_STATIC_LIMIT (and a message
  * on stderr) before anything is launched.  Inputs and outputs are the caller's device buffers,

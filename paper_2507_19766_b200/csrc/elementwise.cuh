@@ -139,7 +139,8 @@ __global__ void seq_entropy_combine_kernel(int n, const int* __restrict__ seq_id
 }
 
 // ------------------------------------------------------------------------------------------
-// Decision stage, one token per thread.
+// Decision stage: four consecutive tokens per thread, 1024 per block, 128-bit loads and stores
+// where the arrays allow it.
 //   MPT (Eq. 9):        A > 0 and logp >= ln tau          gate (Eq. 10): H-bar < sigma
 //   ratio (Eq. 8):      d = logp - old_logp, r = exp(d)   (POIS: r = 1, nothing clipped)
 //   surrogate (Eq. 10): s = min(r A, clip(r, 1 - eps_lo, 1 + eps_hi) A)
@@ -147,6 +148,8 @@ __global__ void seq_entropy_combine_kernel(int n, const int* __restrict__ seq_id
 // Decisions are float32 comparisons against host-computed thresholds; values are float64.
 // ------------------------------------------------------------------------------------------
 constexpr int kDecideThreads = 256;
+constexpr int kDecideVec = 4;
+constexpr int kDecideTokens = kDecideThreads * kDecideVec;
 
 __device__ __forceinline__ int find_sequence(const int* __restrict__ seq_offsets, int S, int t) {
   int lo = 0, hi = S;   // largest i with seq_offsets[i] <= t
@@ -157,6 +160,9 @@ __device__ __forceinline__ int find_sequence(const int* __restrict__ seq_offsets
   return lo;
 }
 
+// kVec: logp, old_logp, segment_version, per-token advantages, grad_coef are 16-byte aligned and flags
+// 4-byte aligned, so a thread's four tokens move as one vector when all four exist.
+template <bool kVec>
 __global__ void decide_kernel(int T, int S, DecideConsts c, const float* __restrict__ logp,
                               const float* __restrict__ old_logp, const int* __restrict__ segment_version,
                               const float* __restrict__ advantages, const int* __restrict__ seq_offsets,
@@ -164,72 +170,128 @@ __global__ void decide_kernel(int T, int S, DecideConsts c, const float* __restr
                               float* __restrict__ grad_coef, uint8_t* __restrict__ flags,
                               DecidePartial* __restrict__ partials) {
   __shared__ double sh_loss[kDecideThreads];
-  __shared__ float sh_abs[kDecideThreads];
-  __shared__ int sh_bucket[kDecideThreads];
+  __shared__ float sh_abs[kDecideTokens];
+  __shared__ signed char sh_bucket[kDecideTokens];
   __shared__ int sh_cnt[5];
   __shared__ int sh_stale[2][ULORL_N_STALENESS];
   const int tid = threadIdx.x;
-  const int t = blockIdx.x * kDecideThreads + tid;
+  const int t0 = blockIdx.x * kDecideTokens + tid * kDecideVec;
   if (tid < 5) sh_cnt[tid] = 0;
   if (tid < ULORL_N_STALENESS) { sh_stale[0][tid] = 0; sh_stale[1][tid] = 0; }
   __syncthreads();
 
+  const bool sais = c.is_mode == ULORL_IS_SAIS;
+  const bool whole = kVec && t0 + kDecideVec <= T;
+  float lp4[kDecideVec], old4[kDecideVec], adv4[kDecideVec];
+  int ver4[kDecideVec];
+#pragma unroll
+  for (int k = 0; k < kDecideVec; ++k) { lp4[k] = 0.f; old4[k] = 0.f; adv4[k] = 0.f; ver4[k] = c.current_version; }
+  if (whole) {
+    const float4 v = *reinterpret_cast<const float4*>(logp + t0);
+    lp4[0] = v.x; lp4[1] = v.y; lp4[2] = v.z; lp4[3] = v.w;
+    if (sais) {
+      const float4 o = *reinterpret_cast<const float4*>(old_logp + t0);
+      old4[0] = o.x; old4[1] = o.y; old4[2] = o.z; old4[3] = o.w;
+    }
+    if (segment_version) {
+      const int4 sv = *reinterpret_cast<const int4*>(segment_version + t0);
+      ver4[0] = sv.x; ver4[1] = sv.y; ver4[2] = sv.z; ver4[3] = sv.w;
+    }
+    if (c.adv_per_token) {
+      const float4 a = *reinterpret_cast<const float4*>(advantages + t0);
+      adv4[0] = a.x; adv4[1] = a.y; adv4[2] = a.z; adv4[3] = a.w;
+    }
+  } else {
+#pragma unroll
+    for (int k = 0; k < kDecideVec; ++k) {
+      const int t = t0 + k;
+      if (t < T) {
+        lp4[k] = logp[t];
+        if (sais) old4[k] = old_logp[t];
+        if (segment_version) ver4[k] = segment_version[t];
+        if (c.adv_per_token) adv4[k] = advantages[t];
+      }
+    }
+  }
+
   double contrib = 0.0;
-  float dabs = 0.f;
-  int bucket = -1;
-  if (t < T) {
-    const int i = find_sequence(seq_offsets, S, t);
-    const float A = c.adv_per_token ? advantages[t] : advantages[i];
-    bool gate = false;
-    if (c.mpt_mode == ULORL_MPT_ALWAYS) {
-      gate = true;
-    } else if (c.mpt_mode == ULORL_MPT_DYNAMIC) {
-      const float h = (c.ent_scope == ULORL_ENT_BATCH) ? *batch_mean : gate_entropy[i];
-      gate = h < c.sigma;
+  float g4[kDecideVec];
+  unsigned f4[kDecideVec];
+  int seq = t0 < T ? find_sequence(seq_offsets, S, t0) : 0;
+#pragma unroll
+  for (int k = 0; k < kDecideVec; ++k) {
+    const int t = t0 + k;
+    float dabs = 0.f;
+    int bucket = -1;
+    g4[k] = 0.f;
+    f4[k] = 0u;
+    if (t < T) {
+      while (seq + 1 < S && seq_offsets[seq + 1] <= t) ++seq;   // the largest i with seq_offsets[i] <= t
+      const int i = seq;
+      const float A = c.adv_per_token ? adv4[k] : advantages[i];
+      bool gate = false;
+      if (c.mpt_mode == ULORL_MPT_ALWAYS) {
+        gate = true;
+      } else if (c.mpt_mode == ULORL_MPT_DYNAMIC) {
+        const float h = (c.ent_scope == ULORL_ENT_BATCH) ? *batch_mean : gate_entropy[i];
+        gate = h < c.sigma;
+      }
+      const float lp = lp4[k];
+      const bool mpt = (A > 0.f) && (lp >= c.ln_tau);
+      const bool msk = mpt && gate;
+      double r = 1.0;
+      bool hi = false, lo = false;
+      if (sais) {
+        const float d = __fsub_rn(lp, old4[k]);
+        r = exp((double)d);
+        hi = (A > 0.f) && (d > c.ln_hi);
+        lo = (A < 0.f) && (d < c.ln_lo);
+        dabs = fabsf(d);
+      }
+      const double Ad = (double)A;
+      const double cl = fmin(fmax(r, 1.0 - c.eps_lo), 1.0 + c.eps_hi);
+      const double s = fmin(r * Ad, cl * Ad);
+      // weight of the token's term: 1/N (Eq. 10), or 1/(G |o_i|) for the per-sample mean of Eq. 5
+      // (inv_N then holds 1/G)
+      double wlen = 1.0;
+      if (c.loss_norm == ULORL_NORM_SEQUENCE) {
+        const int len = seq_offsets[i + 1] - seq_offsets[i];
+        wlen = 1.0 / (double)(len > 0 ? len : 1);
+      }
+      if (!msk) contrib += s * wlen;
+      const double g = (msk || hi || lo) ? 0.0 : -c.inv_N * Ad * r * wlen;
+      g4[k] = (float)g;
+      f4[k] = (msk ? ULORL_FLAG_MASKED : 0u) | (hi ? ULORL_FLAG_CLIP_HIGH : 0u) |
+              (lo ? ULORL_FLAG_CLIP_LOW : 0u) | (mpt ? ULORL_FLAG_MPT : 0u);
+      int st = segment_version ? c.current_version - ver4[k] : 0;
+      st = st < 0 ? 0 : (st > ULORL_N_STALENESS - 1 ? ULORL_N_STALENESS - 1 : st);
+      bucket = st;
+      if (g != 0.0) atomicAdd(&sh_cnt[0], 1);
+      if (mpt) atomicAdd(&sh_cnt[1], 1);
+      if (msk) atomicAdd(&sh_cnt[2], 1);
+      if (hi) atomicAdd(&sh_cnt[3], 1);
+      if (lo) atomicAdd(&sh_cnt[4], 1);
+      atomicAdd(&sh_stale[0][st], 1);
+      if (hi || lo) atomicAdd(&sh_stale[1][st], 1);
     }
-    const float lp = logp[t];
-    const bool mpt = (A > 0.f) && (lp >= c.ln_tau);
-    const bool msk = mpt && gate;
-    double r = 1.0;
-    bool hi = false, lo = false;
-    if (c.is_mode == ULORL_IS_SAIS) {
-      const float d = __fsub_rn(lp, old_logp[t]);
-      r = exp((double)d);
-      hi = (A > 0.f) && (d > c.ln_hi);
-      lo = (A < 0.f) && (d < c.ln_lo);
-      dabs = fabsf(d);
+    sh_abs[tid * kDecideVec + k] = dabs;
+    sh_bucket[tid * kDecideVec + k] = (signed char)bucket;
+  }
+  if (whole) {
+    if (grad_coef) *reinterpret_cast<float4*>(grad_coef + t0) = make_float4(g4[0], g4[1], g4[2], g4[3]);
+    if (flags) *reinterpret_cast<uchar4*>(flags + t0) = make_uchar4((unsigned char)f4[0], (unsigned char)f4[1],
+                                                                    (unsigned char)f4[2], (unsigned char)f4[3]);
+  } else {
+#pragma unroll
+    for (int k = 0; k < kDecideVec; ++k) {
+      const int t = t0 + k;
+      if (t < T) {
+        if (grad_coef) grad_coef[t] = g4[k];
+        if (flags) flags[t] = (uint8_t)f4[k];
+      }
     }
-    const double Ad = (double)A;
-    const double cl = fmin(fmax(r, 1.0 - c.eps_lo), 1.0 + c.eps_hi);
-    const double s = fmin(r * Ad, cl * Ad);
-    // weight of the token's term: 1/N (Eq. 10), or 1/(G |o_i|) for the per-sample mean of Eq. 5
-    // (inv_N then holds 1/G)
-    double wlen = 1.0;
-    if (c.loss_norm == ULORL_NORM_SEQUENCE) {
-      const int len = seq_offsets[i + 1] - seq_offsets[i];
-      wlen = 1.0 / (double)(len > 0 ? len : 1);
-    }
-    if (!msk) contrib = s * wlen;
-    const double g = (msk || hi || lo) ? 0.0 : -c.inv_N * Ad * r * wlen;
-    const float g32 = (float)g;
-    if (grad_coef) grad_coef[t] = g32;
-    const unsigned f = (msk ? ULORL_FLAG_MASKED : 0u) | (hi ? ULORL_FLAG_CLIP_HIGH : 0u) |
-                       (lo ? ULORL_FLAG_CLIP_LOW : 0u) | (mpt ? ULORL_FLAG_MPT : 0u);
-    if (flags) flags[t] = (uint8_t)f;
-    int st = segment_version ? c.current_version - segment_version[t] : 0;
-    st = st < 0 ? 0 : (st > ULORL_N_STALENESS - 1 ? ULORL_N_STALENESS - 1 : st);
-    bucket = st;
-    if (g != 0.0) atomicAdd(&sh_cnt[0], 1);
-    if (mpt) atomicAdd(&sh_cnt[1], 1);
-    if (msk) atomicAdd(&sh_cnt[2], 1);
-    if (hi) atomicAdd(&sh_cnt[3], 1);
-    if (lo) atomicAdd(&sh_cnt[4], 1);
-    atomicAdd(&sh_stale[0][st], 1);
-    if (hi || lo) atomicAdd(&sh_stale[1][st], 1);
   }
   sh_loss[tid] = contrib;
-  sh_abs[tid] = dabs;
-  sh_bucket[tid] = bucket;
   __syncthreads();
   for (int w = kDecideThreads / 2; w > 0; w >>= 1) {
     if (tid < w) sh_loss[tid] += sh_loss[tid + w];
@@ -238,7 +300,7 @@ __global__ void decide_kernel(int T, int S, DecideConsts c, const float* __restr
   DecidePartial* out = partials + blockIdx.x;
   if (tid < ULORL_N_STALENESS) {
     double a = 0.0;
-    for (int k = 0; k < kDecideThreads; ++k)
+    for (int k = 0; k < kDecideTokens; ++k)
       if (sh_bucket[k] == tid) a += (double)sh_abs[k];
     out->stale_abs[tid] = a;
     out->stale_tokens[tid] = sh_stale[0][tid];
@@ -255,73 +317,89 @@ __global__ void decide_kernel(int T, int S, DecideConsts c, const float* __restr
   }
 }
 
-// Sum of the per-block partials in a fixed order; writes the loss and the statistics.
+// Sum of the per-block partials in a fixed order; writes the loss and the statistics.  One pass over the
+// partials with every field in registers, then one fixed butterfly per field inside each warp and a fixed
+// sum over the eight warps: the order of the additions never depends on scheduling.
 constexpr int kFinalThreads = 256;
 
 template <typename V>
-__device__ __forceinline__ V block_sum_fixed(V v, V* sh) {
-  sh[threadIdx.x] = v;
-  __syncthreads();
-  for (int w = kFinalThreads / 2; w > 0; w >>= 1) {
-    if (threadIdx.x < w) sh[threadIdx.x] += sh[threadIdx.x + w];
-    __syncthreads();
-  }
-  V r = sh[0];
-  __syncthreads();
-  return r;
+__device__ __forceinline__ V warp_sum_fixed(V v) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+  return v;
 }
 
 __global__ void finalize_kernel(int T, int n_blocks, double inv_N, const DecidePartial* __restrict__ partials,
                                 const float* __restrict__ batch_mean, const int* __restrict__ status,
                                 float* __restrict__ loss, ulorl_stats_t* __restrict__ stats) {
-  __shared__ double shd[kFinalThreads];
-  __shared__ int shi[kFinalThreads];
-  const int tid = threadIdx.x;
-  double l = 0.0;
-  int cnt[5] = {0, 0, 0, 0, 0};
+  constexpr int kWarps = kFinalThreads / 32;
+  constexpr int kD = 1 + ULORL_N_STALENESS;           // doubles: loss, stale_abs[]
+  constexpr int kI = 5 + 2 * ULORL_N_STALENESS;       // ints: five counters, stale_tokens[], stale_clipped[]
+  __shared__ double shd[kWarps][kD];
+  __shared__ int shi[kWarps][kI];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  double d[kD];
+  int n[kI];
+#pragma unroll
+  for (int k = 0; k < kD; ++k) d[k] = 0.0;
+#pragma unroll
+  for (int k = 0; k < kI; ++k) n[k] = 0;
   for (int b = tid; b < n_blocks; b += kFinalThreads) {
-    l += partials[b].loss_sum;
-    cnt[0] += partials[b].n_active;
-    cnt[1] += partials[b].n_mpt;
-    cnt[2] += partials[b].n_masked;
-    cnt[3] += partials[b].n_clip_high;
-    cnt[4] += partials[b].n_clip_low;
+    const DecidePartial& p = partials[b];
+    d[0] += p.loss_sum;
+    n[0] += p.n_active;
+    n[1] += p.n_mpt;
+    n[2] += p.n_masked;
+    n[3] += p.n_clip_high;
+    n[4] += p.n_clip_low;
+#pragma unroll
+    for (int s = 0; s < ULORL_N_STALENESS; ++s) {
+      d[1 + s] += p.stale_abs[s];
+      n[5 + s] += p.stale_tokens[s];
+      n[5 + ULORL_N_STALENESS + s] += p.stale_clipped[s];
+    }
   }
-  const double loss_sum = block_sum_fixed<double>(l, shd);
-  int tot[5];
-  for (int k = 0; k < 5; ++k) tot[k] = block_sum_fixed<int>(cnt[k], shi);
-  const float loss_value = (float)(-loss_sum * inv_N);
-  if (tid == 0 && loss) loss[0] = loss_value;
+#pragma unroll
+  for (int k = 0; k < kD; ++k) {
+    const double v = warp_sum_fixed<double>(d[k]);
+    if (lane == 0) shd[warp][k] = v;
+  }
+#pragma unroll
+  for (int k = 0; k < kI; ++k) {
+    const int v = warp_sum_fixed<int>(n[k]);
+    if (lane == 0) shi[warp][k] = v;
+  }
+  __syncthreads();
+  if (tid != 0) return;
+  double dt[kD];
+  int nt[kI];
+  for (int k = 0; k < kD; ++k) {
+    dt[k] = 0.0;
+    for (int w = 0; w < kWarps; ++w) dt[k] += shd[w][k];
+  }
+  for (int k = 0; k < kI; ++k) {
+    nt[k] = 0;
+    for (int w = 0; w < kWarps; ++w) nt[k] += shi[w][k];
+  }
+  const float loss_value = (float)(-dt[0] * inv_N);
+  if (loss) loss[0] = loss_value;
   if (!stats) return;
   for (int s = 0; s < ULORL_N_STALENESS; ++s) {
-    double a = 0.0;
-    int nt = 0, nc = 0;
-    for (int b = tid; b < n_blocks; b += kFinalThreads) {
-      a += partials[b].stale_abs[s];
-      nt += partials[b].stale_tokens[s];
-      nc += partials[b].stale_clipped[s];
-    }
-    const double at = block_sum_fixed<double>(a, shd);
-    const int ntt = block_sum_fixed<int>(nt, shi);
-    const int nct = block_sum_fixed<int>(nc, shi);
-    if (tid == 0) {
-      stats->stale_tokens[s] = ntt;
-      stats->stale_clipped[s] = nct;
-      stats->stale_mean_abs_logratio[s] = ntt > 0 ? (float)(at / (double)ntt) : 0.f;
-    }
+    const int ntt = nt[5 + s];
+    stats->stale_tokens[s] = ntt;
+    stats->stale_clipped[s] = nt[5 + ULORL_N_STALENESS + s];
+    stats->stale_mean_abs_logratio[s] = ntt > 0 ? (float)(dt[1 + s] / (double)ntt) : 0.f;
   }
-  if (tid == 0) {
-    stats->loss = loss_value;
-    stats->mean_entropy = *batch_mean;
-    stats->n_tokens = T;
-    stats->n_active = tot[0];
-    stats->n_mpt = tot[1];
-    stats->n_masked = tot[2];
-    stats->n_clip_high = tot[3];
-    stats->n_clip_low = tot[4];
-    stats->device_status = *status;
-    stats->reserved[0] = stats->reserved[1] = stats->reserved[2] = 0;
-  }
+  stats->loss = loss_value;
+  stats->mean_entropy = *batch_mean;
+  stats->n_tokens = T;
+  stats->n_active = nt[0];
+  stats->n_mpt = nt[1];
+  stats->n_masked = nt[2];
+  stats->n_clip_high = nt[3];
+  stats->n_clip_low = nt[4];
+  stats->device_status = *status;
+  stats->reserved[0] = stats->reserved[1] = stats->reserved[2] = 0;
 }
 
 // ------------------------------------------------------------------------------------------

@@ -152,7 +152,7 @@ static Plan make_plan(const ulorl_params_t* p) {
   if (panel < panel_unit) panel = panel_unit;
   pl.panel_tokens = panel;
   pl.dz_ld = pl.tensor ? align_up((size_t)V, 64) : (size_t)V;
-  pl.decide_blocks = (T + kDecideThreads - 1) / kDecideThreads;
+  pl.decide_blocks = (T + kDecideTokens - 1) / kDecideTokens;
   size_t off = 0;
   pl.off_status = off;      off += 256;
   pl.off_batch_mean = pl.off_status + 16;
@@ -376,9 +376,18 @@ static int run_decide(const ulorl_params_t* p, const Plan& pl, const float* logp
   ULORL_LAUNCH_CHECK();
   const DecideConsts c = make_decide_consts(p);
   const float* gate = (p->ent_scope == ULORL_ENT_SUPPLIED) ? entropy_supplied : seq_ent_out;
-  decide_kernel<<<pl.decide_blocks, kDecideThreads, 0, stream>>>(T, S, c, logp, old_logp, segment_version, advantages,
-                                                                  seq_offsets, gate, batch_mean, grad_coef, flags,
-                                                                  partials);
+  // 128-bit accesses when every per-token array starts on a 16-byte boundary (flags: 4 bytes)
+  auto al = [](const void* p, uintptr_t a) { return p == nullptr || (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; };
+  const bool vec = al(logp, 16) && al(old_logp, 16) && al(segment_version, 16) && al(grad_coef, 16) && al(flags, 4) &&
+                   (!p->adv_per_token || al(advantages, 16));
+  if (vec)
+    decide_kernel<true><<<pl.decide_blocks, kDecideThreads, 0, stream>>>(T, S, c, logp, old_logp, segment_version,
+                                                                         advantages, seq_offsets, gate, batch_mean,
+                                                                         grad_coef, flags, partials);
+  else
+    decide_kernel<false><<<pl.decide_blocks, kDecideThreads, 0, stream>>>(T, S, c, logp, old_logp, segment_version,
+                                                                          advantages, seq_offsets, gate, batch_mean,
+                                                                          grad_coef, flags, partials);
   ULORL_LAUNCH_CHECK();
   finalize_kernel<<<1, kFinalThreads, 0, stream>>>(T, pl.decide_blocks, c.inv_N, partials, batch_mean, status, loss,
                                                    reinterpret_cast<ulorl_stats_t*>(stats));
@@ -884,7 +893,7 @@ int ulorl_token_loss_bwd_slabs(const ulorl_params_t* params, const void* hidden,
 //   [256, 256 + 8 * max seqs)      64-bit integer entropy sum per sequence
 //   rest                           one DecidePartial per block of 256 tokens
 constexpr size_t kStaticSeqBytes = sizeof(long long) * (size_t)ULORL_STATIC_MAX_SEQS;
-constexpr size_t kStaticDecideBlocks = ((size_t)ULORL_STATIC_MAX_TOKENS + kDecideThreads - 1) / kDecideThreads;
+constexpr size_t kStaticDecideBlocks = ((size_t)ULORL_STATIC_MAX_TOKENS + kDecideTokens - 1) / kDecideTokens;
 constexpr size_t kStaticScratchBytes = 256 + kStaticSeqBytes + sizeof(DecidePartial) * kStaticDecideBlocks;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
@@ -936,7 +945,7 @@ int ulorl_token_loss_decide_static(const ulorl_params_t* params, const float* lo
   pl.off_batch_mean = 16;
   pl.off_seq_sum = 256;
   pl.off_decide = 256 + kStaticSeqBytes;
-  pl.decide_blocks = (params->T + kDecideThreads - 1) / kDecideThreads;
+  pl.decide_blocks = (params->T + kDecideTokens - 1) / kDecideTokens;
   pl.total = kStaticScratchBytes;
   // the array keeps whatever the previous call left: the status word must start at zero, every
   // other slot that this call reads is written by this call first

@@ -739,3 +739,38 @@ def test_zz_report_colsum_margins():
         print(f"d_W column sums: largest fraction of the statistical bound over {len(COLSUM_MARGINS)} cases = "
               f"{max(COLSUM_MARGINS):.3f}")
         assert max(COLSUM_MARGINS) <= 1.0
+
+
+def test_decision_stage_on_unaligned_arrays_matches_the_vector_path():
+    """The decision kernel moves a thread's four tokens as one 128-bit vector when every per-token array is
+    16-byte aligned; arrays that start one element into an allocation take the scalar accesses.  Same flags,
+    coefficients, loss and statistics, with per-token advantages and a ragged token count."""
+    rng = np.random.default_rng(19)
+    T, S = 4099, 5
+    cuts = np.sort(rng.choice(np.arange(1, T), size=S - 1, replace=False))
+    offsets = torch.from_numpy(np.concatenate([[0], cuts, [T]]).astype(np.int32)).to(DEV)
+    mk = lambda x: torch.from_numpy(x).to(DEV)
+    logp = mk((-np.abs(rng.standard_normal(T + 1)) * 0.02).astype(np.float32))
+    ent = mk((np.abs(rng.standard_normal(T + 1)) * 0.25).astype(np.float32))
+    old = mk((logp.cpu().numpy() + rng.standard_normal(T + 1).astype(np.float32) * 0.15).astype(np.float32))
+    ver = mk(rng.integers(0, 6, size=T + 1).astype(np.int32))
+    adv = mk(rng.choice(np.float32([1.0, -1.0, 0.0, 0.6]), size=T + 1).astype(np.float32))
+    p = B.Params(T=T, H=8, V=16, num_seqs=S, dtype="f32", adv_per_token=True, current_version=5, entropy_target=0.2)
+    outs = []
+    for shift in (0, 1):
+        cut = lambda x: x[1:] if shift else x[1:].clone()          # same values; the clone starts aligned
+        o = B.alloc_fwd_outputs(p, DEV)
+        if shift:
+            o.grad_coef = torch.empty(T + 1, device=DEV)[1:]
+            o.flags = torch.empty(T + 1, dtype=torch.uint8, device=DEV)[1:]
+        outs.append(B.token_loss_decide(p, cut(logp), cut(ent), cut(old), cut(ver), cut(adv), offsets, out=o))
+    torch.cuda.synchronize()
+    a, b = outs
+    assert torch.equal(a.flags, b.flags) and torch.equal(a.grad_coef, b.grad_coef) and torch.equal(a.loss, b.loss)
+    assert a.stats_host() == b.stats_host()
+    ref = O.decide(logp.cpu().numpy()[1:], O.gate_entropy(ent.cpu().numpy()[1:], offsets.cpu().numpy(), "per_seq", None),
+                   old.cpu().numpy()[1:], adv.cpu().numpy()[1:], offsets.cpu().numpy(), ver.cpu().numpy()[1:],
+                   O.OracleParams(current_version=5, entropy_target=0.2), adv_per_token=True)
+    assert np.array_equal(a.flags.cpu().numpy(), ref["flags"])
+    for k in STAT_KEYS:
+        assert a.stats_host()[k] == ref["stats"][k], k
