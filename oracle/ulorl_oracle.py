@@ -71,6 +71,7 @@ class OracleParams:
     loss_norm: str = "tokens"        # "tokens": 1 / sum_i |o_i| (Eq. 7, Eq. 10) | "sequence": (1/G) sum_i 1/|o_i| (Eq. 5)
     norm_seqs: int = 0               # G of Eq. 5 in "sequence" mode; 0 means the sequences of the call
     current_version: int = 0
+    kl_beta: float = 0.0             # beta of Eq. 5's KL-to-reference term; 0 = none (the paper's method, Section 2.3)
 
 
 def _f64(x) -> np.ndarray:
@@ -193,9 +194,21 @@ def decision_thresholds(p: OracleParams):
     return ln_tau, ln_hi, ln_lo
 
 
+def kl_estimate(ref_minus_logp):
+    """Per-token estimate of D_KL[pi_theta || pi_ref] in Eq. 5 from the one generated token:
+    with u = ln pi_ref(o_t) - ln pi_theta(o_t), k = e^u - u - 1.  It is non-negative, zero iff the two
+    log-probs agree, and its mean under o_t ~ pi_theta is the KL divergence (E[e^u] = 1, E[-u] = KL).
+    The paper prints the divergence without an estimator; this is the one of the work Eq. 5 is
+    quoted from."""
+    u = np.asarray(ref_minus_logp, dtype=np.float64)
+    return np.exp(u) - u - 1.0
+
+
 def decide(logp32, gate_ent32, old_logp, advantages, seq_offsets, segment_version,
-           p: OracleParams, adv_per_token: bool = False):
+           p: OracleParams, adv_per_token: bool = False, ref_logp=None):
     """Steps 4-7 on float32 log-probs: mask, ratio, clipped surrogate, loss, d loss/d logp.
+    With p.kl_beta > 0 the token term of Eq. 5 is s_t - beta k_t (k_t = kl_estimate of the token,
+    ref_logp the reference policy's recorded log-prob), inside the mask like the surrogate.
 
     Returns a dict with flags (uint8[T]), ratio, surrogate, grad_coef (float64[T]),
     loss (float64) and the statistics.
@@ -215,11 +228,15 @@ def decide(logp32, gate_ent32, old_logp, advantages, seq_offsets, segment_versio
     eps_hi = float(np.float32(p.clip_eps_high))
     eps_lo = float(np.float32(p.clip_eps_low))
 
+    beta = float(np.float32(p.kl_beta))
+    if beta > 0.0 and ref_logp is None:
+        raise ValueError("kl_beta > 0 needs ref_logp")
     flags = np.zeros(T, dtype=np.uint8)
     ratio = np.ones(T)
     surrogate = np.zeros(T)
     grad_coef = np.zeros(T)
     d_abs = np.zeros(T)
+    kl = np.zeros(T)
     loss_sum = 0.0
     for i in range(S):
         if p.mpt_mode == "always":
@@ -248,9 +265,15 @@ def decide(logp32, gate_ent32, old_logp, advantages, seq_offsets, segment_versio
             c = min(max(r, 1.0 - eps_lo), 1.0 + eps_hi)
             s = min(r * A, c * A)
             keep = 0.0 if msk else 1.0
-            loss_sum += keep * s * wlen
+            # Eq. 5's KL term, when asked for: objective s - beta k, d k / d logp = 1 - e^u
+            dk = 0.0
+            if beta > 0.0:
+                u = float(np.float64(np.float32(ref_logp[t])) - np.float64(logp32[t]))
+                kl[t] = float(kl_estimate(u))
+                dk = 1.0 - float(np.exp(u))
+            loss_sum += keep * (s - beta * kl[t]) * wlen
             # step 7
-            g = -(1.0 / N) * keep * A * r * (0.0 if (hi or lo) else 1.0) * wlen
+            g = -(1.0 / N) * keep * (A * r * (0.0 if (hi or lo) else 1.0) - beta * dk) * wlen
             f = 0
             if msk:
                 f |= FLAG_MASKED
@@ -283,8 +306,9 @@ def decide(logp32, gate_ent32, old_logp, advantages, seq_offsets, segment_versio
         stale_tokens=stale_tokens.astype(np.int64),
         stale_clipped=stale_clipped,
         stale_mean_abs_logratio=np.where(stale_tokens > 0, stale_abs / np.maximum(stale_tokens, 1), 0.0),
+        mean_kl=float(kl.mean()) if T > 0 else 0.0,
     )
-    return dict(flags=flags, ratio=ratio, surrogate=surrogate, grad_coef=grad_coef,
+    return dict(flags=flags, ratio=ratio, surrogate=surrogate, grad_coef=grad_coef, kl=kl,
                 loss=loss, stats=stats)
 
 
@@ -324,7 +348,7 @@ def backward(hidden, W, targets, grad_coef, kappa: float = 1.0, rows=None,
 # --------------------------------------------------------------------------- composition
 def forward(hidden, W, targets, old_logp, segment_version, advantages, seq_offsets,
             p: OracleParams, adv_per_token: bool = False, entropy_supplied=None,
-            rows=None, chunk: int = 256):
+            rows=None, chunk: int = 256, ref_logp=None):
     """Steps 1-7.  With rows=None every token is processed.  The decision stage takes the
     float32 rounding of the float64 log-prob and entropy."""
     logp, ent, lse = token_stats(hidden, W, targets, p.inv_temperature, rows=rows, chunk=chunk)
@@ -336,7 +360,7 @@ def forward(hidden, W, targets, old_logp, segment_version, advantages, seq_offse
     seq_mean, batch_mean = sequence_mean_entropy(ent32, seq_offsets)
     gate32 = gate_entropy(ent32, seq_offsets, p.ent_scope, entropy_supplied)
     dec = decide(logp32, gate32, old_logp, advantages, seq_offsets, segment_version, p,
-                 adv_per_token=adv_per_token)
+                 adv_per_token=adv_per_token, ref_logp=ref_logp)
     out.update(dec)
     out.update(seq_entropy=seq_mean, mean_entropy=batch_mean, gate_entropy=gate32)
     return out
@@ -344,10 +368,10 @@ def forward(hidden, W, targets, old_logp, segment_version, advantages, seq_offse
 
 def fwd_bwd(hidden, W, targets, old_logp, segment_version, advantages, seq_offsets,
             p: OracleParams, adv_per_token: bool = False, entropy_supplied=None,
-            grad_loss: float = 1.0, chunk: int = 256):
+            grad_loss: float = 1.0, chunk: int = 256, ref_logp=None):
     """Steps 1-8 on the whole batch."""
     out = forward(hidden, W, targets, old_logp, segment_version, advantages, seq_offsets, p,
-                  adv_per_token=adv_per_token, entropy_supplied=entropy_supplied, chunk=chunk)
+                  adv_per_token=adv_per_token, entropy_supplied=entropy_supplied, chunk=chunk, ref_logp=ref_logp)
     dH, dW = backward(hidden, W, targets, out["grad_coef"], p.inv_temperature,
                       grad_loss=grad_loss, chunk=chunk)
     out.update(d_hidden=dH, d_W=dW)
@@ -355,7 +379,7 @@ def fwd_bwd(hidden, W, targets, old_logp, segment_version, advantages, seq_offse
 
 
 def objective_value(hidden, W, targets, old_logp, advantages, seq_offsets, masked,
-                    p: OracleParams, adv_per_token: bool = False) -> float:
+                    p: OracleParams, adv_per_token: bool = False, ref_logp=None) -> float:
     """The negated objective of Eq. 10 as a smooth function of (hidden, W) with the mask
     held fixed (the indicator is not differentiated) and everything in float64: used by
     the finite-difference pins.  POIS is evaluated through its defining expression
@@ -380,6 +404,8 @@ def objective_value(hidden, W, targets, old_logp, advantages, seq_offsets, maske
             c = min(max(r, 1.0 - eps_lo), 1.0 + eps_hi)
             if not masked[t]:
                 seq += min(r * A, c * A)
+                if p.kl_beta > 0.0:      # Eq. 5: the token term is s - beta k
+                    seq -= float(np.float32(p.kl_beta)) * float(kl_estimate(float(ref_logp[t]) - logp[t]))
         tot += seq
         if off[i + 1] > off[i]:
             per_sample += seq / float(off[i + 1] - off[i])

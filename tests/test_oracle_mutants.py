@@ -26,13 +26,18 @@ MUTANTS = {
     "strict tau": ("bool(logp32[t] >= ln_tau)", "bool(logp32[t] > ln_tau)"),
     "gate not strict": ("gate = bool(gate_ent32[i] < sigma32)", "gate = bool(gate_ent32[i] <= sigma32)"),
     "normaliser counts unmasked tokens only": ("    loss = -loss_sum / N\n", "    loss = -loss_sum / max(1.0, float(np.count_nonzero((flags & FLAG_MASKED) == 0)))\n"),
-    "clipped tokens keep their gradient": ("g = -(1.0 / N) * keep * A * r * (0.0 if (hi or lo) else 1.0)", "g = -(1.0 / N) * keep * A * r"),
+    "clipped tokens keep their gradient": ("keep * (A * r * (0.0 if (hi or lo) else 1.0) - beta * dk)", "keep * (A * r - beta * dk)"),
     "ratio inverted": ("d32 = np.float32(logp32[t] - np.float32(old_logp[t]))", "d32 = np.float32(np.float32(old_logp[t]) - logp32[t])"),
-    "masked tokens keep their gradient": ("g = -(1.0 / N) * keep * A * r *", "g = -(1.0 / N) * A * r *"),
+    "masked tokens keep their gradient": ("g = -(1.0 / N) * keep * (A * r *", "g = -(1.0 / N) * (A * r *"),
+    "KL term enters with the wrong sign": ("loss_sum += keep * (s - beta * kl[t]) * wlen", "loss_sum += keep * (s + beta * kl[t]) * wlen"),
+    "KL gradient sign": ("dk = 1.0 - float(np.exp(u))", "dk = float(np.exp(u)) - 1.0"),
+    "KL direction reversed": ("u = float(np.float64(np.float32(ref_logp[t])) - np.float64(logp32[t]))", "u = float(np.float64(logp32[t]) - np.float64(np.float32(ref_logp[t])))"),
+    "KL term outside the mask": ("loss_sum += keep * (s - beta * kl[t]) * wlen", "loss_sum += (keep * s - beta * kl[t]) * wlen"),
+    "KL estimate without its linear term": ("return np.exp(u) - u - 1.0", "return np.exp(u) - 1.0"),
     "sample std in the advantages": ("std = (var / G) ** 0.5", "std = (var / (G - 1)) ** 0.5"),
     "advantage sign": ("adv[a + j] = (grp[j] - mean) / std if std > 0 else 0.0", "adv[a + j] = (mean - grp[j]) / std if std > 0 else 0.0"),
     "group filter keeps all-correct groups": ("kept = 0 < n_correct < G", "kept = 0 < n_correct <= G"),
-    "per-sample weight forgotten in the gradient": ("(0.0 if (hi or lo) else 1.0) * wlen", "(0.0 if (hi or lo) else 1.0)"),
+    "per-sample weight forgotten in the gradient": ("- beta * dk) * wlen", "- beta * dk)"),
     "per-sample weight uses T": ("1.0 / max(1.0, float(off[i + 1] - off[i]))", "1.0 / float(T)"),
     "per-sample mode divides by tokens": ("N = float(p.norm_seqs) if p.norm_seqs > 0 else float(S)\n    eps_hi", "N = float(T)\n    eps_hi"),
     "sequence mean divides by T": ("seq_mean[i] = tot / (b - a)", "seq_mean[i] = tot / e.shape[0]"),
@@ -50,11 +55,14 @@ PIN_TESTS = [
     lambda: pins.test_entropy_scopes_and_sequence_means(),
     lambda: pins.test_mean_nll_special_case(),
     lambda: pins.test_dW_column_sums_vanish_and_dhidden_row_form(),
-    lambda: [pins.test_finite_differences(k, "tokens") for k in (1.0, 1.0 / 0.85)],
+    lambda: [pins.test_finite_differences(k, "tokens", 0.0) for k in (1.0, 1.0 / 0.85)],
+    lambda: pins.test_kl_estimate_closed_forms_and_expectation(),
+    lambda: pins.test_kl_term_in_the_decision_stage(),
+    lambda: pins.test_finite_differences(1.0, "tokens", 0.3),
     lambda: pins.test_staleness_statistics(),
     lambda: pins.test_group_advantages_closed_forms(),
     lambda: pins.test_sequence_normalisation_closed_forms(),
-    lambda: pins.test_finite_differences(1.0, "sequence"),
+    lambda: pins.test_finite_differences(1.0, "sequence", 0.0),
 ]
 
 

@@ -439,11 +439,66 @@ def test_dW_column_sums_vanish_and_dhidden_row_form():
     assert np.allclose(out["d_hidden"], expect, atol=1e-12)
 
 
-@pytest.mark.parametrize("kappa,loss_norm", [(1.0, "tokens"), (1.0 / 0.85, "tokens"), (1.0, "sequence")])
-def test_finite_differences(kappa, loss_norm):
-    """Central differences of the Eq. 10 objective in float64 on a tiny problem, with clipped,
-    masked, negative-advantage and zero-advantage tokens present and every token at least
-    1e-2 away from each threshold."""
+def test_kl_estimate_closed_forms_and_expectation():
+    """The per-token KL estimate of Eq. 5's term: zero at u = 0, non-negative, u^2 / 2 to second order, the
+    hand values at u = +-ln 2 (2 - ln 2 - 1 and 1/2 + ln 2 - 1), and its mean under the policy equals the
+    divergence D_KL[pi_theta || pi_ref] (SciPy's rel_entr) for every pair of small categorical distributions."""
+    assert O.kl_estimate(0.0) == 0.0
+    u = np.linspace(-3, 3, 61)
+    assert (O.kl_estimate(u) >= 0).all() and (O.kl_estimate(u)[u != 0] > 0).all()
+    assert abs(O.kl_estimate(1e-4) - 0.5e-8) < 1e-12
+    assert abs(O.kl_estimate(0.6931471805599453) - 0.3068528194400547) < 1e-15
+    assert abs(O.kl_estimate(-0.6931471805599453) - 0.1931471805599453) < 1e-15
+    rng = np.random.default_rng(4)
+    for V in (2, 5, 17):
+        p_theta = rng.dirichlet(np.ones(V))
+        p_ref = rng.dirichlet(np.ones(V))
+        mean_k = float((p_theta * O.kl_estimate(np.log(p_ref) - np.log(p_theta))).sum())
+        assert abs(mean_k - float(scipy.special.rel_entr(p_theta, p_ref).sum())) < 1e-12
+
+
+def test_kl_term_in_the_decision_stage():
+    """Eq. 5's objective s - beta k on hand cases: with A = 0 the loss is +beta k / N and the coefficient
+    beta (1 - e^u) / N (it pulls logp towards the reference); a clipped token keeps the KL gradient; a masked
+    token loses both terms; beta = 0 never reads ref_logp."""
+    one, z = np.float32([1.0]), np.zeros(1, np.int32)
+    ln2 = np.float32(0.6931471805599453)
+    p = O.OracleParams(is_mode="sais", mpt_mode="off", norm_tokens=4, kl_beta=0.5)
+    lp = np.float32([-1.0])
+    out = O.decide(lp, one, lp, np.float32([0.0]), np.array([0, 1]), z, p, ref_logp=lp + ln2)
+    k = 2.0 - float(np.float64(ln2)) - 1.0                       # u = ln 2 as the float32 difference gives it
+    u = float(np.float64(np.float32(lp[0] + ln2)) - np.float64(lp[0]))
+    assert abs(out["kl"][0] - (np.exp(u) - u - 1.0)) < 1e-15 and abs(out["kl"][0] - k) < 1e-6
+    assert abs(out["loss"] - 0.5 * out["kl"][0] / 4) < 1e-15
+    assert abs(out["grad_coef"][0] - 0.5 * (1.0 - np.exp(u)) / 4) < 1e-15 and out["grad_coef"][0] < 0
+    # clipped (ratio e^0.5 > 1.2 with A > 0): the surrogate's gradient is gone, the KL one stays
+    out = O.decide(lp, one, np.float32([-1.5]), one, np.array([0, 1]), z, p, ref_logp=lp - ln2)
+    assert out["flags"][0] & O.FLAG_CLIP_HIGH
+    u = float(np.float64(np.float32(lp[0] - ln2)) - np.float64(lp[0]))
+    assert abs(out["grad_coef"][0] - 0.5 * (1.0 - np.exp(u)) / 4) < 1e-15 and out["grad_coef"][0] > 0
+    assert abs(out["loss"] + (1.2 - 0.5 * out["kl"][0]) / 4) < 1e-8      # 1 + eps with eps = float32(0.2)
+    # masked: nothing of the token is left
+    pm = O.OracleParams(is_mode="sais", mpt_mode="always", norm_tokens=4, kl_beta=0.5)
+    hi_lp = np.float32([-0.001])
+    out = O.decide(hi_lp, one, hi_lp, one, np.array([0, 1]), z, pm, ref_logp=hi_lp - ln2)
+    assert out["flags"][0] & O.FLAG_MASKED and out["loss"] == 0.0 and out["grad_coef"][0] == 0.0
+    assert out["stats"]["mean_kl"] > 0            # the diagnostic still sees the token
+    # beta = 0: the reference is not needed
+    p0 = O.OracleParams(is_mode="sais", mpt_mode="off", norm_tokens=4)
+    a = O.decide(lp, one, lp, one, np.array([0, 1]), z, p0)
+    b = O.decide(lp, one, lp, one, np.array([0, 1]), z, p0, ref_logp=lp - ln2)
+    assert a["loss"] == b["loss"] and a["grad_coef"][0] == b["grad_coef"][0] and b["stats"]["mean_kl"] == 0.0
+    with pytest.raises(ValueError):
+        O.decide(lp, one, lp, one, np.array([0, 1]), z, p)
+
+
+@pytest.mark.parametrize("kappa,loss_norm,kl_beta", [(1.0, "tokens", 0.0), (1.0 / 0.85, "tokens", 0.0),
+                                                    (1.0, "sequence", 0.0), (1.0, "tokens", 0.3),
+                                                    (1.0 / 0.85, "sequence", 0.3)])
+def test_finite_differences(kappa, loss_norm, kl_beta):
+    """Central differences of the Eq. 10 objective (with Eq. 5's KL term when kl_beta > 0) in float64 on a
+    tiny problem, with clipped, masked, negative-advantage and zero-advantage tokens present and every
+    token at least 1e-2 away from each threshold."""
     T, H, V = 6, 4, 10
     rng = np.random.default_rng(23)
     hidden = rng.standard_normal((T, H))
@@ -460,17 +515,18 @@ def test_finite_differences(kappa, loss_norm):
     shift = np.array([0.0, 0.4, -0.1, -0.5, 0.15, 0.0])     # clip-high on 1, clip-low on 3
     old = (logp - shift).astype(np.float32)
     p = O.OracleParams(is_mode="sais", mpt_mode="always", inv_temperature=kappa, norm_tokens=9, loss_norm=loss_norm,
-                       norm_seqs=4)
-    out = O.fwd_bwd(hidden, W, targets, old, np.zeros(T, np.int32), adv, offsets, p)
+                       norm_seqs=4, kl_beta=kl_beta)
+    ref = (logp + np.array([0.3, -0.2, 0.5, -0.4, 0.1, 0.25])).astype(np.float32)
+    out = O.fwd_bwd(hidden, W, targets, old, np.zeros(T, np.int32), adv, offsets, p, ref_logp=ref)
     fl = out["flags"]
     assert fl[0] & O.FLAG_MASKED and fl[1] & O.FLAG_CLIP_HIGH and fl[3] & O.FLAG_CLIP_LOW
-    assert out["stats"]["n_active"] == 2
+    assert out["stats"]["n_active"] == (2 if kl_beta == 0 else 5)   # the KL gradient also flows through clipped and A = 0 tokens
     ln_tau, ln_hi, ln_lo = O.decision_thresholds(p)
     d = logp - old
     assert (np.abs(d - ln_hi) > 1e-2).all() and (np.abs(d - ln_lo) > 1e-2).all()
     assert (np.abs(logp - ln_tau) > 1e-2).all()
     masked = (fl & O.FLAG_MASKED) != 0
-    f = lambda h, w: O.objective_value(h, w, targets, old, adv, offsets, masked, p)
+    f = lambda h, w: O.objective_value(h, w, targets, old, adv, offsets, masked, p, ref_logp=ref)
     # the oracle takes d from float32 log-probs, the smooth objective from float64 ones:
     # values agree to float32 rounding of logp (1e-7 relative), nothing coarser
     assert abs(f(hidden, W) - out["loss"]) < 1e-7
