@@ -103,6 +103,9 @@ typedef struct {
   int32_t dw_dtype;            /* ulorl_dtype_t of d_W: F32 (default), or BF16 -- the sum over tokens is then    */
                                /* still taken in float32 (in the workspace, which grows by 4 V H bytes) and      */
                                /* rounded once when a row of d_W is final.  Part of the workspace size.          */
+  float kl_beta;               /* beta of the KL-to-reference term of Eq. 5; 0 (the paper's method, Section 2.3:  */
+                               /* the term is removed) leaves ref_logp unread.  With beta > 0 the token term is   */
+                               /* s_t - beta k_t, k_t = e^u - u - 1, u = ref_logp[t] - logp[t], inside the mask.  */
 } ulorl_params_t;
 
 typedef struct {
@@ -113,7 +116,8 @@ typedef struct {
   int32_t stale_clipped[ULORL_N_STALENESS];    /* of which clipped                                                */
   float stale_mean_abs_logratio[ULORL_N_STALENESS];
   int32_t device_status;       /* copy of the workspace status word at the end of the forward call                */
-  int32_t reserved[3];
+  float mean_kl;               /* token mean of the KL estimate k_t over the call (0 when kl_beta = 0)            */
+  int32_t reserved[2];
 } ulorl_stats_t;
 
 /* Bytes of workspace both calls need for these params (pure host function; 0 on invalid params). */
@@ -125,6 +129,8 @@ size_t ulorl_workspace_bytes(const ulorl_params_t* params);
  *   targets [T] int32      generated token ids y_t
  *   old_logp [T] f32       log-prob recorded at rollout by the policy that generated the token's
  *                          segment (Eq. 8); may be NULL in POIS mode
+ *   ref_logp [T] f32       log-prob of the token under the reference policy of Eq. 5's KL term; read only
+ *                          when kl_beta > 0, else may be NULL
  *   segment_version [T]    id of that policy (statistics only); may be NULL
  *   advantages             f32, [num_seqs] or [T] (adv_per_token)
  *   seq_offsets [S+1]      int32, non-decreasing, seq_offsets[0] = 0, seq_offsets[S] = T
@@ -135,7 +141,7 @@ size_t ulorl_workspace_bytes(const ulorl_params_t* params);
  */
 int ulorl_token_loss_fwd(const ulorl_params_t* params,
                          const void* hidden, const void* W, const int32_t* targets,
-                         const float* old_logp, const int32_t* segment_version,
+                         const float* old_logp, const float* ref_logp, const int32_t* segment_version,
                          const float* advantages, const int32_t* seq_offsets,
                          const float* entropy_supplied,
                          float* logp, float* entropy, float* lse, float* grad_coef,
@@ -149,7 +155,7 @@ int ulorl_token_loss_fwd(const ulorl_params_t* params,
  */
 int ulorl_token_loss_decide(const ulorl_params_t* params,
                             const float* logp, const float* entropy,
-                            const float* old_logp, const int32_t* segment_version,
+                            const float* old_logp, const float* ref_logp, const int32_t* segment_version,
                             const float* advantages, const int32_t* seq_offsets,
                             const float* entropy_supplied,
                             float* grad_coef, uint8_t* flags, float* seq_entropy, float* loss,
@@ -184,7 +190,7 @@ int ulorl_token_loss_decide(const ulorl_params_t* params,
 #define ULORL_STATIC_MAX_SEQS   (1 << 16)
 int ulorl_token_loss_decide_static(const ulorl_params_t* params,
                                    const float* logp, const float* entropy,
-                                   const float* old_logp, const int32_t* segment_version,
+                                   const float* old_logp, const float* ref_logp, const int32_t* segment_version,
                                    const float* advantages, const int32_t* seq_offsets,
                                    const float* entropy_supplied,
                                    float* grad_coef, uint8_t* flags, float* seq_entropy, float* loss,
@@ -316,7 +322,7 @@ int ulorl_kernel_timing_end(float* total_ms, int64_t* launches);
 size_t ulorl_host_step_arena_bytes(const ulorl_params_t* params);
 int ulorl_token_loss_step_host(const ulorl_params_t* params,
                                const void* h_hidden, const void* h_W, const int32_t* h_targets,
-                               const float* h_old_logp, const int32_t* h_segment_version,
+                               const float* h_old_logp, const float* h_ref_logp, const int32_t* h_segment_version,
                                const float* h_advantages, const int32_t* h_seq_offsets,
                                const float* h_entropy_supplied,
                                float* h_logp, float* h_entropy, uint8_t* h_flags, float* h_seq_entropy,

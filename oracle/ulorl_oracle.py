@@ -273,7 +273,7 @@ def decide(logp32, gate_ent32, old_logp, advantages, seq_offsets, segment_versio
                 dk = 1.0 - float(np.exp(u))
             loss_sum += keep * (s - beta * kl[t]) * wlen
             # step 7
-            g = -(1.0 / N) * keep * (A * r * (0.0 if (hi or lo) else 1.0) - beta * dk) * wlen
+            g = -(1.0 / N) * keep * (A * r * (0.0 if (hi or lo) else 1.0) - beta * dk) * wlen + 0.0   # + 0.0: no -0
             f = 0
             if msk:
                 f |= FLAG_MASKED

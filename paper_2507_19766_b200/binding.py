@@ -46,7 +46,7 @@ class CParams(ctypes.Structure):
         ("norm_tokens", ctypes.c_int64), ("current_version", ctypes.c_int32),
         ("dw_accumulate", ctypes.c_int32), ("kernel_path", ctypes.c_int32), ("bwd_panel_tokens", ctypes.c_int32),
         ("compact_rows", ctypes.c_int32), ("loss_norm", ctypes.c_int32), ("norm_seqs", ctypes.c_int32),
-        ("dw_dtype", ctypes.c_int32),
+        ("dw_dtype", ctypes.c_int32), ("kl_beta", ctypes.c_float),
     ]
 
 
@@ -57,7 +57,7 @@ class CStats(ctypes.Structure):
         ("n_masked", ctypes.c_int32), ("n_clip_high", ctypes.c_int32), ("n_clip_low", ctypes.c_int32),
         ("stale_tokens", ctypes.c_int32 * N_STALENESS), ("stale_clipped", ctypes.c_int32 * N_STALENESS),
         ("stale_mean_abs_logratio", ctypes.c_float * N_STALENESS),
-        ("device_status", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3),
+        ("device_status", ctypes.c_int32), ("mean_kl", ctypes.c_float), ("reserved", ctypes.c_int32 * 2),
     ]
 
 
@@ -88,11 +88,11 @@ def load_library() -> ctypes.CDLL:
     lib.ulorl_workspace_bytes.restype = ctypes.c_size_t
     lib.ulorl_workspace_bytes.argtypes = [cp]
     lib.ulorl_token_loss_fwd.restype = ctypes.c_int
-    lib.ulorl_token_loss_fwd.argtypes = [cp] + [vp] * 16 + [vp, ctypes.c_size_t, vp]
+    lib.ulorl_token_loss_fwd.argtypes = [cp] + [vp] * 17 + [vp, ctypes.c_size_t, vp]
     lib.ulorl_token_loss_decide.restype = ctypes.c_int
-    lib.ulorl_token_loss_decide.argtypes = [cp] + [vp] * 12 + [vp, ctypes.c_size_t, vp]
+    lib.ulorl_token_loss_decide.argtypes = [cp] + [vp] * 13 + [vp, ctypes.c_size_t, vp]
     lib.ulorl_token_loss_decide_static.restype = ctypes.c_int
-    lib.ulorl_token_loss_decide_static.argtypes = [cp] + [vp] * 12 + [vp]
+    lib.ulorl_token_loss_decide_static.argtypes = [cp] + [vp] * 13 + [vp]
     lib.ulorl_group_advantages.restype = ctypes.c_int
     lib.ulorl_group_advantages.argtypes = [vp, ctypes.c_int32, ctypes.c_int32, vp, vp, vp]
     lib.ulorl_sequence_entropy_partials.restype = ctypes.c_int
@@ -120,7 +120,7 @@ def load_library() -> ctypes.CDLL:
     lib.ulorl_host_step_arena_bytes.restype = ctypes.c_size_t
     lib.ulorl_host_step_arena_bytes.argtypes = [cp]
     lib.ulorl_token_loss_step_host.restype = ctypes.c_int
-    lib.ulorl_token_loss_step_host.argtypes = [cp] + [vp] * 16 + [vp, ctypes.c_size_t, vp]
+    lib.ulorl_token_loss_step_host.argtypes = [cp] + [vp] * 17 + [vp, ctypes.c_size_t, vp]
     _lib = lib
     return lib
 
@@ -160,6 +160,7 @@ class Params:
     loss_norm: str = "tokens"
     norm_seqs: int = 0
     dw_dtype: str = "f32"
+    kl_beta: float = 0.0
 
     @property
     def dw_torch_dtype(self):
@@ -171,7 +172,8 @@ class Params:
                        self.clip_eps_low, self.clip_eps_high, self.mpt_tau, self.entropy_target,
                        self.inv_temperature, self.norm_tokens, self.current_version, int(self.dw_accumulate),
                        _PATH[self.kernel_path], self.bwd_panel_tokens, int(self.compact_rows),
-                       _NORM[self.loss_norm], self.norm_seqs, BF16 if self.dw_dtype == "bf16" else F32)
+                       _NORM[self.loss_norm], self.norm_seqs, BF16 if self.dw_dtype == "bf16" else F32,
+                       self.kl_beta)
 
 
 def workspace_bytes(p: Params) -> int:
@@ -230,7 +232,8 @@ def decode_stats(stats: torch.Tensor) -> dict:
     return dict(loss=s.loss, mean_entropy=s.mean_entropy, n_tokens=s.n_tokens, n_active=s.n_active, n_mpt=s.n_mpt,
                 n_masked=s.n_masked, n_clip_high=s.n_clip_high, n_clip_low=s.n_clip_low,
                 stale_tokens=list(s.stale_tokens), stale_clipped=list(s.stale_clipped),
-                stale_mean_abs_logratio=list(s.stale_mean_abs_logratio), device_status=s.device_status)
+                stale_mean_abs_logratio=list(s.stale_mean_abs_logratio), device_status=s.device_status,
+                mean_kl=s.mean_kl)
 
 
 def alloc_workspace(p: Params, device) -> torch.Tensor:
@@ -246,7 +249,8 @@ def alloc_fwd_outputs(p: Params, device) -> FwdOut:
 
 
 def token_loss_fwd(p: Params, hidden, W, targets, old_logp, segment_version, advantages, seq_offsets,
-                   entropy_supplied=None, out: Optional[FwdOut] = None, workspace: Optional[torch.Tensor] = None) -> FwdOut:
+                   entropy_supplied=None, out: Optional[FwdOut] = None, workspace: Optional[torch.Tensor] = None,
+                   ref_logp=None) -> FwdOut:
     """ulorl_token_loss_fwd on the current CUDA stream."""
     lib = load_library()
     dev = hidden.device
@@ -263,7 +267,8 @@ def token_loss_fwd(p: Params, hidden, W, targets, old_logp, segment_version, adv
     out = out or alloc_fwd_outputs(p, dev)
     workspace = workspace if workspace is not None else alloc_workspace(p, dev)
     code = lib.ulorl_token_loss_fwd(
-        ctypes.byref(p.to_c()), _ptr(hidden), _ptr(W), _ptr(targets), _ptr(old_logp), _ptr(segment_version),
+        ctypes.byref(p.to_c()), _ptr(hidden), _ptr(W), _ptr(targets), _ptr(old_logp), _ptr(ref_logp),
+        _ptr(segment_version),
         _ptr(advantages), _ptr(seq_offsets), _ptr(entropy_supplied), _ptr(out.logp), _ptr(out.entropy), _ptr(out.lse),
         _ptr(out.grad_coef), _ptr(out.flags), _ptr(out.seq_entropy), _ptr(out.loss), _ptr(out.stats),
         _ptr(workspace), workspace.numel(), _stream())
@@ -273,7 +278,7 @@ def token_loss_fwd(p: Params, hidden, W, targets, old_logp, segment_version, adv
 
 def token_loss_decide(p: Params, logp, entropy, old_logp, segment_version, advantages, seq_offsets,
                       entropy_supplied=None, out: Optional[FwdOut] = None,
-                      workspace: Optional[torch.Tensor] = None) -> FwdOut:
+                      workspace: Optional[torch.Tensor] = None, ref_logp=None) -> FwdOut:
     """ulorl_token_loss_decide: the elementwise stage on given per-token log-probs and entropies."""
     lib = load_library()
     dev = logp.device
@@ -283,7 +288,8 @@ def token_loss_decide(p: Params, logp, entropy, old_logp, segment_version, advan
     out.logp, out.entropy = logp, entropy
     workspace = workspace if workspace is not None else alloc_workspace(p, dev)
     code = lib.ulorl_token_loss_decide(
-        ctypes.byref(p.to_c()), _ptr(logp), _ptr(entropy), _ptr(old_logp), _ptr(segment_version), _ptr(advantages),
+        ctypes.byref(p.to_c()), _ptr(logp), _ptr(entropy), _ptr(old_logp), _ptr(ref_logp), _ptr(segment_version),
+        _ptr(advantages),
         _ptr(seq_offsets), _ptr(entropy_supplied), _ptr(out.grad_coef), _ptr(out.flags), _ptr(out.seq_entropy),
         _ptr(out.loss), _ptr(out.stats), _ptr(workspace), workspace.numel(), _stream())
     _check(code, "ulorl_token_loss_decide")
@@ -291,7 +297,7 @@ def token_loss_decide(p: Params, logp, entropy, old_logp, segment_version, advan
 
 
 def token_loss_decide_static(p: Params, logp, entropy, old_logp, segment_version, advantages, seq_offsets,
-                             entropy_supplied=None, out: Optional[FwdOut] = None) -> FwdOut:
+                             entropy_supplied=None, out: Optional[FwdOut] = None, ref_logp=None) -> FwdOut:
     """ulorl_token_loss_decide_static: the elementwise stage with no workspace argument, for callers
     that cannot allocate device memory; its scratch is a fixed array inside the library (at most
     STATIC_MAX_TOKENS tokens and STATIC_MAX_SEQS sequences).  `out` must be given by such a caller;
@@ -302,7 +308,8 @@ def token_loss_decide_static(p: Params, logp, entropy, old_logp, segment_version
     out = out or alloc_fwd_outputs(p, logp.device)
     out.logp, out.entropy = logp, entropy
     code = lib.ulorl_token_loss_decide_static(
-        ctypes.byref(p.to_c()), _ptr(logp), _ptr(entropy), _ptr(old_logp), _ptr(segment_version), _ptr(advantages),
+        ctypes.byref(p.to_c()), _ptr(logp), _ptr(entropy), _ptr(old_logp), _ptr(ref_logp), _ptr(segment_version),
+        _ptr(advantages),
         _ptr(seq_offsets), _ptr(entropy_supplied), _ptr(out.grad_coef), _ptr(out.flags), _ptr(out.seq_entropy),
         _ptr(out.loss), _ptr(out.stats), _stream())
     _check(code, "ulorl_token_loss_decide_static")
@@ -383,12 +390,12 @@ def _hptr(t: Optional[torch.Tensor]):
 
 def token_loss_step_host(p: Params, arena: torch.Tensor, hidden, W, targets, old_logp, segment_version, advantages,
                          seq_offsets, entropy_supplied=None, logp=None, entropy=None, flags=None, seq_entropy=None,
-                         loss=None, stats=None, d_hidden=None, d_W=None):
+                         loss=None, stats=None, d_hidden=None, d_W=None, ref_logp=None):
     """ulorl_token_loss_step_host: every tensor except `arena` lives in host memory (pinned for
     asynchronous copies).  Asynchronous on the current stream."""
     code = load_library().ulorl_token_loss_step_host(
-        ctypes.byref(p.to_c()), _hptr(hidden), _hptr(W), _hptr(targets), _hptr(old_logp), _hptr(segment_version),
-        _hptr(advantages), _hptr(seq_offsets), _hptr(entropy_supplied), _hptr(logp), _hptr(entropy), _hptr(flags),
+        ctypes.byref(p.to_c()), _hptr(hidden), _hptr(W), _hptr(targets), _hptr(old_logp), _hptr(ref_logp),
+        _hptr(segment_version), _hptr(advantages), _hptr(seq_offsets), _hptr(entropy_supplied), _hptr(logp), _hptr(entropy), _hptr(flags),
         _hptr(seq_entropy), _hptr(loss), _hptr(stats), _hptr(d_hidden), _hptr(d_W), _ptr(arena), arena.numel(),
         _stream())
     _check(code, "ulorl_token_loss_step_host")

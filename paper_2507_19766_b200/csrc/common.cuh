@@ -21,6 +21,7 @@ constexpr int kStatusBadOffsets = 4;   // seq_offsets not 0 = o[0] <= o[1] <= ..
 // so that the loss and the statistics do not depend on scheduling.
 struct DecidePartial {
   double loss_sum;
+  double kl_sum;
   double stale_abs[ULORL_N_STALENESS];
   int n_active, n_mpt, n_masked, n_clip_high, n_clip_low, pad;
   int stale_tokens[ULORL_N_STALENESS];
@@ -31,7 +32,7 @@ struct DecidePartial {
 // roundings of float64 evaluations, so that no transcendental sits inside a comparison.
 struct DecideConsts {
   float ln_tau, ln_hi, ln_lo, sigma;
-  double eps_lo, eps_hi, inv_N;
+  double eps_lo, eps_hi, inv_N, kl_beta;
   int is_mode, mpt_mode, ent_scope, adv_per_token, current_version, loss_norm;
 };
 

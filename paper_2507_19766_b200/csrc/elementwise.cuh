@@ -164,12 +164,14 @@ __device__ __forceinline__ int find_sequence(const int* __restrict__ seq_offsets
 // 4-byte aligned, so a thread's four tokens move as one vector when all four exist.
 template <bool kVec>
 __global__ void decide_kernel(int T, int S, DecideConsts c, const float* __restrict__ logp,
-                              const float* __restrict__ old_logp, const int* __restrict__ segment_version,
+                              const float* __restrict__ old_logp, const float* __restrict__ ref_logp,
+                              const int* __restrict__ segment_version,
                               const float* __restrict__ advantages, const int* __restrict__ seq_offsets,
                               const float* __restrict__ gate_entropy, const float* __restrict__ batch_mean,
                               float* __restrict__ grad_coef, uint8_t* __restrict__ flags,
                               DecidePartial* __restrict__ partials) {
   __shared__ double sh_loss[kDecideThreads];
+  __shared__ double sh_kl[kDecideThreads];
   __shared__ float sh_abs[kDecideTokens];
   __shared__ signed char sh_bucket[kDecideTokens];
   __shared__ int sh_cnt[5];
@@ -181,17 +183,22 @@ __global__ void decide_kernel(int T, int S, DecideConsts c, const float* __restr
   __syncthreads();
 
   const bool sais = c.is_mode == ULORL_IS_SAIS;
+  const bool with_kl = c.kl_beta > 0.0;
   const bool whole = kVec && t0 + kDecideVec <= T;
-  float lp4[kDecideVec], old4[kDecideVec], adv4[kDecideVec];
+  float lp4[kDecideVec], old4[kDecideVec], adv4[kDecideVec], ref4[kDecideVec];
   int ver4[kDecideVec];
 #pragma unroll
-  for (int k = 0; k < kDecideVec; ++k) { lp4[k] = 0.f; old4[k] = 0.f; adv4[k] = 0.f; ver4[k] = c.current_version; }
+  for (int k = 0; k < kDecideVec; ++k) { lp4[k] = 0.f; old4[k] = 0.f; adv4[k] = 0.f; ref4[k] = 0.f; ver4[k] = c.current_version; }
   if (whole) {
     const float4 v = *reinterpret_cast<const float4*>(logp + t0);
     lp4[0] = v.x; lp4[1] = v.y; lp4[2] = v.z; lp4[3] = v.w;
     if (sais) {
       const float4 o = *reinterpret_cast<const float4*>(old_logp + t0);
       old4[0] = o.x; old4[1] = o.y; old4[2] = o.z; old4[3] = o.w;
+    }
+    if (with_kl) {
+      const float4 rf = *reinterpret_cast<const float4*>(ref_logp + t0);
+      ref4[0] = rf.x; ref4[1] = rf.y; ref4[2] = rf.z; ref4[3] = rf.w;
     }
     if (segment_version) {
       const int4 sv = *reinterpret_cast<const int4*>(segment_version + t0);
@@ -208,13 +215,14 @@ __global__ void decide_kernel(int T, int S, DecideConsts c, const float* __restr
       if (t < T) {
         lp4[k] = logp[t];
         if (sais) old4[k] = old_logp[t];
+        if (with_kl) ref4[k] = ref_logp[t];
         if (segment_version) ver4[k] = segment_version[t];
         if (c.adv_per_token) adv4[k] = advantages[t];
       }
     }
   }
 
-  double contrib = 0.0;
+  double contrib = 0.0, kl_acc = 0.0;
   float g4[kDecideVec];
   unsigned f4[kDecideVec];
   int seq = t0 < T ? find_sequence(seq_offsets, S, t0) : 0;
@@ -258,8 +266,18 @@ __global__ void decide_kernel(int T, int S, DecideConsts c, const float* __restr
         const int len = seq_offsets[i + 1] - seq_offsets[i];
         wlen = 1.0 / (double)(len > 0 ? len : 1);
       }
-      if (!msk) contrib += s * wlen;
-      const double g = (msk || hi || lo) ? 0.0 : -c.inv_N * Ad * r * wlen;
+      // Eq. 5's KL-to-reference term, when asked for: token term s - beta k with k = e^u - u - 1,
+      // u = ref_logp - logp (exact in float64), d k / d logp = 1 - e^u; inside the mask like the surrogate
+      double k_t = 0.0, dk = 0.0;
+      if (with_kl) {
+        const double u = (double)ref4[k] - (double)lp;
+        const double eu = exp(u);
+        k_t = eu - u - 1.0;
+        dk = 1.0 - eu;
+        kl_acc += k_t;
+      }
+      if (!msk) contrib += (s - c.kl_beta * k_t) * wlen;
+      const double g = msk ? 0.0 : -c.inv_N * (((hi || lo) ? 0.0 : Ad * r) - c.kl_beta * dk) * wlen + 0.0;   // + 0.0: no -0
       g4[k] = (float)g;
       f4[k] = (msk ? ULORL_FLAG_MASKED : 0u) | (hi ? ULORL_FLAG_CLIP_HIGH : 0u) |
               (lo ? ULORL_FLAG_CLIP_LOW : 0u) | (mpt ? ULORL_FLAG_MPT : 0u);
@@ -292,9 +310,10 @@ __global__ void decide_kernel(int T, int S, DecideConsts c, const float* __restr
     }
   }
   sh_loss[tid] = contrib;
+  sh_kl[tid] = kl_acc;
   __syncthreads();
   for (int w = kDecideThreads / 2; w > 0; w >>= 1) {
-    if (tid < w) sh_loss[tid] += sh_loss[tid + w];
+    if (tid < w) { sh_loss[tid] += sh_loss[tid + w]; sh_kl[tid] += sh_kl[tid + w]; }
     __syncthreads();
   }
   DecidePartial* out = partials + blockIdx.x;
@@ -308,6 +327,7 @@ __global__ void decide_kernel(int T, int S, DecideConsts c, const float* __restr
   }
   if (tid == 0) {
     out->loss_sum = sh_loss[0];
+    out->kl_sum = sh_kl[0];
     out->n_active = sh_cnt[0];
     out->n_mpt = sh_cnt[1];
     out->n_masked = sh_cnt[2];
@@ -333,7 +353,7 @@ __global__ void finalize_kernel(int T, int n_blocks, double inv_N, const DecideP
                                 const float* __restrict__ batch_mean, const int* __restrict__ status,
                                 float* __restrict__ loss, ulorl_stats_t* __restrict__ stats) {
   constexpr int kWarps = kFinalThreads / 32;
-  constexpr int kD = 1 + ULORL_N_STALENESS;           // doubles: loss, stale_abs[]
+  constexpr int kD = 2 + ULORL_N_STALENESS;           // doubles: loss, stale_abs[], KL sum (last)
   constexpr int kI = 5 + 2 * ULORL_N_STALENESS;       // ints: five counters, stale_tokens[], stale_clipped[]
   __shared__ double shd[kWarps][kD];
   __shared__ int shi[kWarps][kI];
@@ -347,6 +367,7 @@ __global__ void finalize_kernel(int T, int n_blocks, double inv_N, const DecideP
   for (int b = tid; b < n_blocks; b += kFinalThreads) {
     const DecidePartial& p = partials[b];
     d[0] += p.loss_sum;
+    d[kD - 1] += p.kl_sum;
     n[0] += p.n_active;
     n[1] += p.n_mpt;
     n[2] += p.n_masked;
@@ -399,7 +420,8 @@ __global__ void finalize_kernel(int T, int n_blocks, double inv_N, const DecideP
   stats->n_clip_high = nt[3];
   stats->n_clip_low = nt[4];
   stats->device_status = *status;
-  stats->reserved[0] = stats->reserved[1] = stats->reserved[2] = 0;
+  stats->mean_kl = T > 0 ? (float)(dt[kD - 1] / (double)T) : 0.f;
+  stats->reserved[0] = stats->reserved[1] = 0;
 }
 
 // ------------------------------------------------------------------------------------------

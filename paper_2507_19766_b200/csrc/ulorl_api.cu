@@ -96,6 +96,7 @@ static int validate_params(const ulorl_params_t* p) {
   if (p->norm_tokens < 0 || p->bwd_panel_tokens < 0) return ULORL_ERR_INVALID_ARG;
   if (p->compact_rows != 0 && p->compact_rows != 1) return ULORL_ERR_INVALID_ARG;
   if (p->dw_dtype != ULORL_F32 && p->dw_dtype != ULORL_BF16) return ULORL_ERR_INVALID_ARG;
+  if (!(p->kl_beta >= 0.f) || !std::isfinite(p->kl_beta)) return ULORL_ERR_INVALID_ARG;
   if (p->H % 8 != 0) return ULORL_ERR_UNSUPPORTED;
   // the exact integer entropy sums hold 2^29 nats; no token's entropy exceeds ln V
   if ((double)p->T * std::log((double)p->V + 1.0) >= kEntropyFixCapacity) return ULORL_ERR_UNSUPPORTED;
@@ -356,11 +357,13 @@ static DecideConsts make_decide_consts(const ulorl_params_t* p) {
   c.adv_per_token = p->adv_per_token;
   c.current_version = p->current_version;
   c.loss_norm = p->loss_norm;
+  c.kl_beta = (double)p->kl_beta;
   return c;
 }
 
 static int run_decide(const ulorl_params_t* p, const Plan& pl, const float* logp, const float* entropy,
-                      const float* old_logp, const int32_t* segment_version, const float* advantages,
+                      const float* old_logp, const float* ref_logp, const int32_t* segment_version,
+                      const float* advantages,
                       const int32_t* seq_offsets, const float* entropy_supplied, float* grad_coef, uint8_t* flags,
                       float* seq_entropy, float* loss, void* stats, uint8_t* ws, cudaStream_t stream) {
   const int T = p->T, S = p->num_seqs;
@@ -379,15 +382,15 @@ static int run_decide(const ulorl_params_t* p, const Plan& pl, const float* logp
   // 128-bit accesses when every per-token array starts on a 16-byte boundary (flags: 4 bytes)
   auto al = [](const void* p, uintptr_t a) { return p == nullptr || (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; };
   const bool vec = al(logp, 16) && al(old_logp, 16) && al(segment_version, 16) && al(grad_coef, 16) && al(flags, 4) &&
-                   (!p->adv_per_token || al(advantages, 16));
+                   (!p->adv_per_token || al(advantages, 16)) && (!(p->kl_beta > 0.f) || al(ref_logp, 16));
   if (vec)
-    decide_kernel<true><<<pl.decide_blocks, kDecideThreads, 0, stream>>>(T, S, c, logp, old_logp, segment_version,
-                                                                         advantages, seq_offsets, gate, batch_mean,
-                                                                         grad_coef, flags, partials);
+    decide_kernel<true><<<pl.decide_blocks, kDecideThreads, 0, stream>>>(T, S, c, logp, old_logp, ref_logp,
+                                                                         segment_version, advantages, seq_offsets, gate,
+                                                                         batch_mean, grad_coef, flags, partials);
   else
-    decide_kernel<false><<<pl.decide_blocks, kDecideThreads, 0, stream>>>(T, S, c, logp, old_logp, segment_version,
-                                                                          advantages, seq_offsets, gate, batch_mean,
-                                                                          grad_coef, flags, partials);
+    decide_kernel<false><<<pl.decide_blocks, kDecideThreads, 0, stream>>>(T, S, c, logp, old_logp, ref_logp,
+                                                                          segment_version, advantages, seq_offsets, gate,
+                                                                          batch_mean, grad_coef, flags, partials);
   ULORL_LAUNCH_CHECK();
   finalize_kernel<<<1, kFinalThreads, 0, stream>>>(T, pl.decide_blocks, c.inv_N, partials, batch_mean, status, loss,
                                                    reinterpret_cast<ulorl_stats_t*>(stats));
@@ -395,11 +398,13 @@ static int run_decide(const ulorl_params_t* p, const Plan& pl, const float* logp
   return ULORL_OK;
 }
 
-static int validate_decide_args(const ulorl_params_t* p, const float* old_logp, const float* advantages,
+static int validate_decide_args(const ulorl_params_t* p, const float* old_logp, const float* ref_logp,
+                                const float* advantages,
                                 const int32_t* seq_offsets, const float* entropy_supplied, float* seq_entropy,
                                 float* loss) {
   if (!advantages || !seq_offsets || !loss || !seq_entropy) return ULORL_ERR_INVALID_ARG;
   if (p->is_mode == ULORL_IS_SAIS && !old_logp) return ULORL_ERR_INVALID_ARG;
+  if (p->kl_beta > 0.f && !ref_logp) return ULORL_ERR_INVALID_ARG;
   if (p->mpt_mode == ULORL_MPT_DYNAMIC && p->ent_scope == ULORL_ENT_SUPPLIED && !entropy_supplied)
     return ULORL_ERR_INVALID_ARG;
   return ULORL_OK;
@@ -505,7 +510,8 @@ int ulorl_check_status(void* workspace, void* cuda_stream) {
 }
 
 int ulorl_token_loss_decide(const ulorl_params_t* params, const float* logp, const float* entropy,
-                            const float* old_logp, const int32_t* segment_version, const float* advantages,
+                            const float* old_logp, const float* ref_logp, const int32_t* segment_version,
+                            const float* advantages,
                             const int32_t* seq_offsets, const float* entropy_supplied, float* grad_coef,
                             uint8_t* flags, float* seq_entropy, float* loss, void* stats, void* workspace,
                             size_t workspace_bytes, void* cuda_stream) {
@@ -514,18 +520,19 @@ int ulorl_token_loss_decide(const ulorl_params_t* params, const float* logp, con
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (params->T == 0) return empty_forward(workspace, workspace_bytes, loss, stats, stream);
   if (!logp || !entropy || !workspace) return ULORL_ERR_INVALID_ARG;
-  st = validate_decide_args(params, old_logp, advantages, seq_offsets, entropy_supplied, seq_entropy, loss);
+  st = validate_decide_args(params, old_logp, ref_logp, advantages, seq_offsets, entropy_supplied, seq_entropy, loss);
   if (st != ULORL_OK) return st;
   const Plan pl = make_plan(params);
   if (workspace_bytes < pl.total) return ULORL_ERR_WORKSPACE;
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
   if (cudaMemsetAsync(ws + pl.off_status, 0, 256, stream) != cudaSuccess) return ULORL_ERR_CUDA;
-  return run_decide(params, pl, logp, entropy, old_logp, segment_version, advantages, seq_offsets, entropy_supplied,
+  return run_decide(params, pl, logp, entropy, old_logp, ref_logp, segment_version, advantages, seq_offsets, entropy_supplied,
                     grad_coef, flags, seq_entropy, loss, stats, ws, stream);
 }
 
 static int fwd_impl(const ulorl_params_t* params, const void* hidden, const void* W, const int32_t* targets,
-                    const float* old_logp, const int32_t* segment_version, const float* advantages,
+                    const float* old_logp, const float* ref_logp, const int32_t* segment_version,
+                    const float* advantages,
                     const int32_t* seq_offsets, const float* entropy_supplied, float* logp, float* entropy,
                     float* lse, float* grad_coef, uint8_t* flags, float* seq_entropy, float* loss, void* stats,
                     void* workspace, size_t workspace_bytes, void* cuda_stream, const StepHooks* hooks) {
@@ -534,7 +541,7 @@ static int fwd_impl(const ulorl_params_t* params, const void* hidden, const void
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (params->T == 0) return empty_forward(workspace, workspace_bytes, loss, stats, stream);
   if (!hidden || !W || !targets || !logp || !entropy || !lse || !workspace) return ULORL_ERR_INVALID_ARG;
-  st = validate_decide_args(params, old_logp, advantages, seq_offsets, entropy_supplied, seq_entropy, loss);
+  st = validate_decide_args(params, old_logp, ref_logp, advantages, seq_offsets, entropy_supplied, seq_entropy, loss);
   if (st != ULORL_OK) return st;
   if (!aligned16(hidden) || !aligned16(W) || !aligned16(workspace)) return ULORL_ERR_UNSUPPORTED;
   const Plan pl = make_plan(params);
@@ -620,16 +627,17 @@ static int fwd_impl(const ulorl_params_t* params, const void* hidden, const void
                                                              lse);
     ULORL_LAUNCH_CHECK();
   }
-  return run_decide(params, pl, logp, entropy, old_logp, segment_version, advantages, seq_offsets, entropy_supplied,
+  return run_decide(params, pl, logp, entropy, old_logp, ref_logp, segment_version, advantages, seq_offsets, entropy_supplied,
                     grad_coef, flags, seq_entropy, loss, stats, ws, stream);
 }
 
 int ulorl_token_loss_fwd(const ulorl_params_t* params, const void* hidden, const void* W, const int32_t* targets,
-                         const float* old_logp, const int32_t* segment_version, const float* advantages,
+                         const float* old_logp, const float* ref_logp, const int32_t* segment_version,
+                         const float* advantages,
                          const int32_t* seq_offsets, const float* entropy_supplied, float* logp, float* entropy,
                          float* lse, float* grad_coef, uint8_t* flags, float* seq_entropy, float* loss, void* stats,
                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
-  return fwd_impl(params, hidden, W, targets, old_logp, segment_version, advantages, seq_offsets, entropy_supplied, logp,
+  return fwd_impl(params, hidden, W, targets, old_logp, ref_logp, segment_version, advantages, seq_offsets, entropy_supplied, logp,
                   entropy, lse, grad_coef, flags, seq_entropy, loss, stats, workspace, workspace_bytes, cuda_stream,
                   nullptr);
 }
@@ -920,7 +928,8 @@ static int static_scratch_address(uint8_t** out) {
 }
 
 int ulorl_token_loss_decide_static(const ulorl_params_t* params, const float* logp, const float* entropy,
-                                   const float* old_logp, const int32_t* segment_version, const float* advantages,
+                                   const float* old_logp, const float* ref_logp, const int32_t* segment_version,
+                                   const float* advantages,
                                    const int32_t* seq_offsets, const float* entropy_supplied, float* grad_coef,
                                    uint8_t* flags, float* seq_entropy, float* loss, void* stats, void* cuda_stream) {
   int st = validate_params(params);
@@ -938,7 +947,7 @@ int ulorl_token_loss_decide_static(const ulorl_params_t* params, const float* lo
   if (st != ULORL_OK) return st;
   if (params->T == 0) return empty_forward(ws, 256, loss, stats, stream);
   if (!logp || !entropy) return ULORL_ERR_INVALID_ARG;
-  st = validate_decide_args(params, old_logp, advantages, seq_offsets, entropy_supplied, seq_entropy, loss);
+  st = validate_decide_args(params, old_logp, ref_logp, advantages, seq_offsets, entropy_supplied, seq_entropy, loss);
   if (st != ULORL_OK) return st;
   Plan pl{};
   pl.off_status = 0;
@@ -950,7 +959,7 @@ int ulorl_token_loss_decide_static(const ulorl_params_t* params, const float* lo
   // the array keeps whatever the previous call left: the status word must start at zero, every
   // other slot that this call reads is written by this call first
   if (cudaMemsetAsync(ws + pl.off_status, 0, 256, stream) != cudaSuccess) return ULORL_ERR_CUDA;
-  return run_decide(params, pl, logp, entropy, old_logp, segment_version, advantages, seq_offsets, entropy_supplied,
+  return run_decide(params, pl, logp, entropy, old_logp, ref_logp, segment_version, advantages, seq_offsets, entropy_supplied,
                     grad_coef, flags, seq_entropy, loss, stats, ws, stream);
 }
 
@@ -1028,7 +1037,7 @@ int ulorl_kernel_timing_end(float* total_ms, int64_t* launches) {
 // ------------------------------------------------------------------ host-buffer step
 namespace {
 struct HostStepLayout {
-  size_t hidden, W, targets, old_logp, segver, adv, seq_off, ent_sup;
+  size_t hidden, W, targets, old_logp, ref_logp, segver, adv, seq_off, ent_sup;
   size_t logp, entropy, lse, grad_coef, flags, seq_entropy, loss, stats, d_hidden, d_W, ws, total;
   size_t elem;
 };
@@ -1088,6 +1097,7 @@ HostStepLayout host_step_layout(const ulorl_params_t* p) {
   L.W = take(V * H * L.elem);
   L.targets = take(T * 4);
   L.old_logp = take(T * 4);
+  L.ref_logp = take(p->kl_beta > 0.f ? T * 4 : 0);
   L.segver = take(T * 4);
   L.adv = take((p->adv_per_token ? T : S) * 4);
   L.seq_off = take((S + 1) * 4);
@@ -1114,7 +1124,8 @@ size_t ulorl_host_step_arena_bytes(const ulorl_params_t* params) {
 }
 
 int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidden, const void* h_W,
-                               const int32_t* h_targets, const float* h_old_logp, const int32_t* h_segment_version,
+                               const int32_t* h_targets, const float* h_old_logp, const float* h_ref_logp,
+                               const int32_t* h_segment_version,
                                const float* h_advantages, const int32_t* h_seq_offsets,
                                const float* h_entropy_supplied, float* h_logp, float* h_entropy, uint8_t* h_flags,
                                float* h_seq_entropy, float* h_loss, void* h_stats, void* h_d_hidden, void* h_d_W,
@@ -1141,6 +1152,7 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
     return (!src || !bytes) ? cudaSuccess : cudaMemcpyAsync(a + off, src, bytes, cudaMemcpyHostToDevice, hs->in);
   };
   if (!ok(h2d(L.targets, h_targets, T * 4)) || !ok(h2d(L.old_logp, h_old_logp, T * 4)) ||
+      !ok(h2d(L.ref_logp, h_ref_logp, T * 4)) ||
       !ok(h2d(L.segver, h_segment_version, T * 4)) ||
       !ok(h2d(L.adv, h_advantages, (params->adv_per_token ? T : S) * 4)) ||
       !ok(h2d(L.seq_off, h_seq_offsets, (S + 1) * 4)) || !ok(h2d(L.ent_sup, h_entropy_supplied, S * 4)))
@@ -1247,6 +1259,7 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
   }
   st = fwd_impl(params, a + L.hidden, a + L.W, reinterpret_cast<const int32_t*>(a + L.targets),
                 h_old_logp ? reinterpret_cast<const float*>(a + L.old_logp) : nullptr,
+                h_ref_logp ? reinterpret_cast<const float*>(a + L.ref_logp) : nullptr,
                 h_segment_version ? reinterpret_cast<const int32_t*>(a + L.segver) : nullptr,
                 reinterpret_cast<const float*>(a + L.adv), reinterpret_cast<const int32_t*>(a + L.seq_off),
                 h_entropy_supplied ? reinterpret_cast<const float*>(a + L.ent_sup) : nullptr,

@@ -18,7 +18,8 @@ def both_params(batch: synth.Batch, **over):
     wl = batch.workload
     kw = dict(is_mode=wl.is_mode, mpt_mode=wl.mpt_mode, ent_scope="per_seq", clip_eps_low=wl.clip_eps_low,
               clip_eps_high=wl.clip_eps_high, mpt_tau=wl.mpt_tau, entropy_target=wl.entropy_target,
-              inv_temperature=1.0, norm_tokens=0, current_version=batch.current_version, loss_norm="tokens", norm_seqs=0)
+              inv_temperature=1.0, norm_tokens=0, current_version=batch.current_version, loss_norm="tokens", norm_seqs=0,
+              kl_beta=0.0)
     extra = {k: over.pop(k) for k in list(over) if k in ("kernel_path", "bwd_panel_tokens", "dw_accumulate",
                                                          "adv_per_token", "compact_rows")}
     kw.update(over)

@@ -774,3 +774,89 @@ def test_decision_stage_on_unaligned_arrays_matches_the_vector_path():
     assert np.array_equal(a.flags.cpu().numpy(), ref["flags"])
     for k in STAT_KEYS:
         assert a.stats_host()[k] == ref["stats"][k], k
+
+
+# --------------------------------------------------------------------------- KL-to-reference term of Eq. 5
+def kl_reference(batch, seed):
+    """A recorded reference log-prob per token: the rollout record moved by N(0, 0.3)."""
+    rng = np.random.default_rng(seed)
+    return (batch.old_logp.numpy() + 0.3 * rng.standard_normal(batch.workload.T).astype(np.float32)).astype(np.float32)
+
+
+@pytest.mark.parametrize("path,loss_norm", [("tensor", "tokens"), ("simt", "sequence")])
+def test_kl_term_matches_the_oracle(path, loss_norm):
+    """Eq. 5's objective s - beta k through the whole path: forward (loss, coefficients, mean KL) and both
+    gradients against the oracle; the decision kernel on the oracle's float32 log-probs to 2e-6."""
+    wl = synth.WORKLOADS["small"].scaled(T=700, S=5, H=328, V=3001, lengths="lognormal:100:400", segment_len=64,
+                                         planted=0.3, beta_planted=(80.0, 160.0), mpt_mode="always")
+    batch = synth.make_batch(wl, seed=5)
+    ref_lp = kl_reference(batch, 77)
+    gp, op = both_params(batch, kernel_path=path, kl_beta=0.25, loss_norm=loss_norm)
+    oi = oracle_inputs(batch)
+    ref = O.fwd_bwd(oi["hidden"], oi["W"], oi["targets"], oi["old_logp"], oi["segment_version"], oi["advantages"],
+                    oi["seq_offsets"], op, ref_logp=ref_lp)
+    b = batch.to(DEV)
+    rl = torch.from_numpy(ref_lp).to(DEV)
+    ws = B.alloc_workspace(gp, DEV)
+    out = B.token_loss_fwd(gp, b.hidden, b.W, b.targets, b.old_logp, b.segment_version, b.advantages, b.seq_offsets,
+                           workspace=ws, ref_logp=rl)
+    torch.cuda.synchronize()
+    near = near_threshold(ref["logp"], oi["old_logp"], ref["seq_entropy"], oi["seq_offsets"], op)
+    differ = out.flags.cpu().numpy() != ref["flags"]
+    assert not (differ & ~near).any()
+    st = out.stats_host()
+    assert abs(st["mean_kl"] - ref["stats"]["mean_kl"]) <= 1e-3 * max(ref["stats"]["mean_kl"], 1e-3)
+    assert ref["stats"]["mean_kl"] > 0.01 and ref["stats"]["n_clip_high"] + ref["stats"]["n_clip_low"] > 0
+    # the oracle's float32 log-probs through the decision kernel: same decisions, coefficients and loss to float32
+    t32 = lambda x: torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(DEV)
+    dec = B.token_loss_decide(gp, t32(ref["logp"]), t32(ref["entropy"]), b.old_logp, b.segment_version, b.advantages,
+                              b.seq_offsets, ref_logp=rl)
+    assert np.array_equal(dec.flags.cpu().numpy(), ref["flags"])
+    assert np.allclose(dec.grad_coef.cpu().numpy(), ref["grad_coef"], rtol=2e-6, atol=1e-12)
+    assert abs(float(dec.loss.cpu()[0]) - ref["loss"]) <= 2e-6 * max(1.0, abs(ref["loss"]))
+    assert abs(dec.stats_host()["mean_kl"] - ref["stats"]["mean_kl"]) <= 1e-6
+    assert dec.stats_host()["n_active"] == ref["stats"]["n_active"]
+    # clipped tokens are active now (their KL gradient flows); masked ones are not
+    clipped = (ref["flags"] & (O.FLAG_CLIP_HIGH | O.FLAG_CLIP_LOW)) != 0
+    masked = (ref["flags"] & O.FLAG_MASKED) != 0
+    g = dec.grad_coef.cpu().numpy()
+    assert (g[clipped & ~masked] != 0).all() and (g[masked] == 0).all()
+    # backward on the oracle's coefficients
+    dH, dW = B.token_loss_bwd(gp, b.hidden, b.W, b.targets, out.lse, t32(ref["grad_coef"]), workspace=ws)
+    torch.cuda.synchronize()
+    assert rel_l2(dH.float().cpu().numpy(), ref["d_hidden"]) <= TOL_GRAD
+    assert rel_l2(dW.cpu().numpy(), ref["d_W"]) <= TOL_GRAD
+    if not differ.any():
+        assert abs(float(out.loss.cpu()[0]) - ref["loss"]) <= TOL_LOSS * max(abs(ref["loss"]), 1e-3)
+    # beta > 0 without a reference is refused; beta = 0 ignores one
+    with pytest.raises(B.UlorlError):
+        B.token_loss_fwd(gp, b.hidden, b.W, b.targets, b.old_logp, b.segment_version, b.advantages, b.seq_offsets,
+                         workspace=ws)
+    gp0, _ = both_params(batch, kernel_path=path, loss_norm=loss_norm)
+    a0 = B.token_loss_fwd(gp0, b.hidden, b.W, b.targets, b.old_logp, b.segment_version, b.advantages, b.seq_offsets)
+    a1 = B.token_loss_fwd(gp0, b.hidden, b.W, b.targets, b.old_logp, b.segment_version, b.advantages, b.seq_offsets,
+                          ref_logp=rl)
+    assert torch.equal(a0.grad_coef, a1.grad_coef) and torch.equal(a0.loss, a1.loss) and a1.stats_host()["mean_kl"] == 0.0
+
+
+def test_kl_term_through_the_host_buffer_step():
+    wl = synth.WORKLOADS["small"].scaled(T=900, S=4, H=256, V=2500, lengths="tiny", planted=0.3,
+                                         beta_planted=(100.0, 200.0), mpt_mode="always")
+    batch = synth.make_batch(wl, seed=41)
+    ref_lp = kl_reference(batch, 78)
+    gp, _ = both_params(batch, kl_beta=0.1)
+    b = batch.to(DEV)
+    ws = B.alloc_workspace(gp, DEV)
+    out = B.token_loss_fwd(gp, b.hidden, b.W, b.targets, b.old_logp, b.segment_version, b.advantages, b.seq_offsets,
+                           workspace=ws, ref_logp=torch.from_numpy(ref_lp).to(DEV))
+    dH, dW = B.token_loss_bwd(gp, b.hidden, b.W, b.targets, out.lse, out.grad_coef, workspace=ws)
+    arena = torch.empty(B.host_step_arena_bytes(gp), dtype=torch.uint8, device=DEV)
+    pin = lambda t: t.contiguous().pin_memory()
+    ho = dict(loss=torch.empty(1).pin_memory(), stats=torch.empty(out.stats.numel(), dtype=torch.uint8).pin_memory(),
+              d_hidden=torch.empty(wl.T, wl.H, dtype=torch.bfloat16).pin_memory(), d_W=torch.empty(wl.V, wl.H).pin_memory())
+    B.token_loss_step_host(gp, arena, pin(batch.hidden), pin(batch.W), pin(batch.targets), pin(batch.old_logp),
+                           pin(batch.segment_version), pin(batch.advantages), pin(batch.seq_offsets),
+                           ref_logp=pin(torch.from_numpy(ref_lp)), **ho)
+    torch.cuda.synchronize()
+    assert torch.equal(ho["loss"], out.loss.cpu()) and torch.equal(ho["d_W"], dW.cpu()) and torch.equal(ho["d_hidden"], dH.cpu())
+    assert B.decode_stats(ho["stats"]) == out.stats_host() and out.stats_host()["mean_kl"] > 0

@@ -33,8 +33,8 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_struct_sizes_match_header(lib):
-    # 9 int32 + 5 float + (pad) int64 + 5 int32 (+ pad)
-    assert ctypes.sizeof(B.CParams) == 96
+    # 9 int32 + 5 float + (pad) int64 + 8 int32 + 1 float (+ pad)
+    assert ctypes.sizeof(B.CParams) == 104
     assert ctypes.sizeof(B.CStats) == 4 * (2 + 6 + 3 * 16 + 4)
 
 
@@ -62,7 +62,7 @@ def test_status_strings(lib):
 
 def test_null_arguments_are_rejected_without_a_device(lib):
     p = B.Params(T=8, H=64, V=128, num_seqs=1).to_c()
-    args = [None] * 16
+    args = [None] * 17
     code = lib.ulorl_token_loss_fwd(ctypes.byref(p), *args, None, 0, None)
     assert code == -1
     code = lib.ulorl_token_loss_bwd(ctypes.byref(p), *([None] * 8), None, 0, None)

@@ -37,7 +37,7 @@ MUTANTS = {
     "sample std in the advantages": ("std = (var / G) ** 0.5", "std = (var / (G - 1)) ** 0.5"),
     "advantage sign": ("adv[a + j] = (grp[j] - mean) / std if std > 0 else 0.0", "adv[a + j] = (mean - grp[j]) / std if std > 0 else 0.0"),
     "group filter keeps all-correct groups": ("kept = 0 < n_correct < G", "kept = 0 < n_correct <= G"),
-    "per-sample weight forgotten in the gradient": ("- beta * dk) * wlen", "- beta * dk)"),
+    "per-sample weight forgotten in the gradient": ("- beta * dk) * wlen + 0.0", "- beta * dk) + 0.0"),
     "per-sample weight uses T": ("1.0 / max(1.0, float(off[i + 1] - off[i]))", "1.0 / float(T)"),
     "per-sample mode divides by tokens": ("N = float(p.norm_seqs) if p.norm_seqs > 0 else float(S)\n    eps_hi", "N = float(T)\n    eps_hi"),
     "sequence mean divides by T": ("seq_mean[i] = tot / (b - a)", "seq_mean[i] = tot / e.shape[0]"),

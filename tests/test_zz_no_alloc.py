@@ -71,6 +71,6 @@ def test_static_scratch_variant_rejects_batches_beyond_its_limit():
     lib = B.load_library()
     for T, S in ((B.STATIC_MAX_TOKENS + 1, 1), (B.STATIC_MAX_SEQS + 1, B.STATIC_MAX_SEQS + 1)):
         p = B.Params(T=T, H=8, V=16, num_seqs=S, dtype="f32").to_c()
-        code = lib.ulorl_token_loss_decide_static(ctypes.byref(p), *([None] * 12), None)
+        code = lib.ulorl_token_loss_decide_static(ctypes.byref(p), *([None] * 13), None)
         assert code == -7
     assert "scratch" in B.status_string(-7)
