@@ -442,6 +442,9 @@ struct StepHooks {
   // Tensor path: when set, the last panel computes d_W before d_hidden and in slabs of vocabulary rows,
   // and this is called after each slab (first row, rows): those rows of d_W are final from then on.
   std::function<int(int, int)> after_dw_slab;
+  // Tensor path, with after_dw_slab: device memory for a second dz panel (same size as the workspace's), or
+  // NULL.  With it the last two panels are reordered so that more work follows the point where d_W is final.
+  void* dz_second_buffer = nullptr;
 };
 
 }  // namespace ulorl
@@ -734,69 +737,95 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
     CUtensorMap map_dw_out;   // d_W as the target of 128-row x 32-column float tiles
     st = make_map(&map_dw_out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, d_W, (uint64_t)V, (uint64_t)H, (uint64_t)H, 32, kBM);
     if (st != ULORL_OK) return st;
-    CUtensorMap map_dz_out;   // the dz panel (all its rows) as the target of 128-row x 64-column bf16 tiles
-    st = make_map_bf16(&map_dz_out, dz, (uint64_t)pl.panel_tokens, (uint64_t)pl.dz_ld, (uint64_t)pl.dz_ld, 64, kBM);
-    if (st != ULORL_OK) return st;
+    // One token panel: its rows, its dz buffer and the tensor maps over that buffer.
+    struct Panel {
+      int t0, rows, index;
+      CUtensorMap dz_out, dz_k, dz_mn;
+    };
+    auto make_panel = [&](int t0, int index, __nv_bfloat16* buf, Panel& pn) -> int {
+      pn.t0 = t0;
+      pn.rows = (T - t0) < pl.panel_tokens ? (T - t0) : pl.panel_tokens;
+      pn.index = index;
+      // the whole buffer as the target of 128-row x 64-column bf16 tiles; its valid rows as the operand of the
+      // two gradient contractions (K-major for d_hidden, MN-major for d_W)
+      int rc = make_map_bf16(&pn.dz_out, buf, (uint64_t)pl.panel_tokens, (uint64_t)pl.dz_ld, (uint64_t)pl.dz_ld, 64, kBM);
+      if (rc != ULORL_OK) return rc;
+      rc = make_map_bf16(&pn.dz_k, buf, (uint64_t)pn.rows, (uint64_t)pl.dz_ld, (uint64_t)pl.dz_ld, kBK, kBM);
+      if (rc != ULORL_OK) return rc;
+      return make_map_bf16(&pn.dz_mn, buf, (uint64_t)pn.rows, (uint64_t)pl.dz_ld, (uint64_t)pl.dz_ld, 64, kBK);
+    };
+    // dz panel: recompute logits, softmax minus one-hot scaled by the token's coefficient
+    auto run_dz = [&](const Panel& pn) -> int {
+      UmmaArgs a{};
+      a.M = pn.rows; a.N = V; a.K = H;
+      a.m_tiles = (pn.rows + tile_m - 1) / tile_m;
+      a.n_tiles = (int)(pl.dz_ld / kBN) + ((pl.dz_ld % kBN) ? 1 : 0);
+      a.group_m = kRasterGroup;
+      a.a_mn0 = pn.t0;
+      a.row0 = pn.t0;
+      a.kappa = kappa;
+      a.targets = targets; a.lse = lse; a.grad_coef = grad_coef; a.grad_loss = grad_loss;
+      a.dz_cols = (int)pl.dz_ld;
+      a.dyn_rows = n_active; a.dyn_base = pn.t0;
+      a.status = status;
+      return launch_umma<kModeDz>(pl, map_hidden_k, map_w_k, pn.dz_out, a, stream);
+    };
+    // d_hidden[t0 + m, h] = sum_v dz[m, v] W[v, h]
+    auto run_d_hidden = [&](const Panel& pn) -> int {
+      UmmaArgs a{};
+      a.M = pn.rows; a.N = H; a.K = V;
+      a.m_tiles = (pn.rows + tile_m - 1) / tile_m;
+      a.n_tiles = (H + grad_unit_cols(pl) - 1) / grad_unit_cols(pl);
+      a.group_m = kGradRasterGroup;
+      a.row0 = pn.t0;
+      a.d_hidden = static_cast<__nv_bfloat16*>(d_hidden_out);
+      a.out_ld = (size_t)H;
+      a.dyn_rows = n_active; a.dyn_base = pn.t0;
+      a.status = status;
+      int rc = launch_umma<kModeDHidden>(pl, pn.dz_k, map_w_mn, map_w_mn, a, stream);
+      if (rc != ULORL_OK) return rc;
+      if (hooks && hooks->after_dhidden_panel && !pl.compact) return hooks->after_dhidden_panel(pn.t0, pn.rows);
+      return ULORL_OK;
+    };
+    // d_W[v, h] (+)= sum_m dz[m, v] hidden[t0 + m, h] for the vocabulary rows [v0, v0 + v_rows)
+    auto run_d_W = [&](const Panel& pn, int v0, int v_rows) -> int {
+      UmmaArgs a{};
+      a.M = v_rows; a.N = H; a.K = pn.rows;
+      a.m_tiles = (v_rows + tile_m - 1) / tile_m;
+      a.n_tiles = (H + grad_unit_cols(pl) - 1) / grad_unit_cols(pl);
+      a.group_m = kGradRasterGroup;
+      a.a_mn0 = v0;
+      a.b_k0 = pn.t0;
+      a.row0 = v0;
+      a.d_W = d_W;
+      a.out_ld = (size_t)H;
+      a.accumulate = (pn.index > 0 || acc_into || pl.compact) ? 1 : 0;
+      a.dyn_rows = n_active; a.dyn_base = pn.t0;
+      a.status = status;
+      return launch_umma<kModeDW>(pl, pn.dz_mn, map_hidden_mn, map_dw_out, a, stream);
+    };
+    const int n_panels = (T + pl.panel_tokens - 1) / pl.panel_tokens;
+    const bool by_slabs = hooks && hooks->after_dw_slab;
+    // With a second dz buffer from the caller, the d_hidden contraction of the panel before the last is put off
+    // until d_W is final: the last two panels then run dz, d_W, dz', d_W' (slab by slab), d_hidden, d_hidden', so
+    // that two d_hidden contractions, not one, are still to come while the rows of d_W are already on their way out.
+    __nv_bfloat16* dz_alt = (hooks && by_slabs && !pl.compact && n_panels >= 2)
+                                ? static_cast<__nv_bfloat16*>(hooks->dz_second_buffer) : nullptr;
+    Panel held{};
     for (int t0 = 0, panel = 0; t0 < T; t0 += pl.panel_tokens, ++panel) {
-      const int rows = (T - t0) < pl.panel_tokens ? (T - t0) : pl.panel_tokens;
-      // dz panel: recompute logits, softmax minus one-hot scaled by the token's coefficient
-      {
-        UmmaArgs a{};
-        a.M = rows; a.N = V; a.K = H;
-        a.m_tiles = (rows + tile_m - 1) / tile_m;
-        a.n_tiles = (int)(pl.dz_ld / kBN) + ((pl.dz_ld % kBN) ? 1 : 0);
-        a.group_m = kRasterGroup;
-        a.a_mn0 = t0;
-        a.row0 = t0;
-        a.kappa = kappa;
-        a.targets = targets; a.lse = lse; a.grad_coef = grad_coef; a.grad_loss = grad_loss;
-        a.dz_cols = (int)pl.dz_ld;
-        a.dyn_rows = n_active; a.dyn_base = t0;
-        a.status = status;
-        st = launch_umma<kModeDz>(pl, map_hidden_k, map_w_k, map_dz_out, a, stream);
+      const bool last_panel = panel == n_panels - 1;
+      Panel pn;
+      st = make_panel(t0, panel, (dz_alt && last_panel) ? dz_alt : dz, pn);
+      if (st != ULORL_OK) return st;
+      st = run_dz(pn);
+      if (st != ULORL_OK) return st;
+      if (dz_alt && panel == n_panels - 2) {       // its d_hidden follows the last panel's d_W
+        st = run_d_W(pn, 0, V);
         if (st != ULORL_OK) return st;
+        held = pn;
+        continue;
       }
-      CUtensorMap map_dz_k, map_dz_mn;
-      st = make_map_bf16(&map_dz_k, dz, (uint64_t)rows, (uint64_t)pl.dz_ld, (uint64_t)pl.dz_ld, kBK, kBM);
-      if (st != ULORL_OK) return st;
-      st = make_map_bf16(&map_dz_mn, dz, (uint64_t)rows, (uint64_t)pl.dz_ld, (uint64_t)pl.dz_ld, 64, kBK);
-      if (st != ULORL_OK) return st;
-      // d_hidden[t0 + m, h] = sum_v dz[m, v] W[v, h]
-      auto run_d_hidden = [&]() -> int {
-        UmmaArgs a{};
-        a.M = rows; a.N = H; a.K = V;
-        a.m_tiles = (rows + tile_m - 1) / tile_m;
-        a.n_tiles = (H + grad_unit_cols(pl) - 1) / grad_unit_cols(pl);
-        a.group_m = kGradRasterGroup;
-        a.row0 = t0;
-        a.d_hidden = static_cast<__nv_bfloat16*>(d_hidden_out);
-        a.out_ld = (size_t)H;
-        a.dyn_rows = n_active; a.dyn_base = t0;
-        a.status = status;
-        int rc = launch_umma<kModeDHidden>(pl, map_dz_k, map_w_mn, map_w_mn, a, stream);
-        if (rc != ULORL_OK) return rc;
-        if (hooks && hooks->after_dhidden_panel && !pl.compact) return hooks->after_dhidden_panel(t0, rows);
-        return ULORL_OK;
-      };
-      // d_W[v, h] (+)= sum_m dz[m, v] hidden[t0 + m, h] for the vocabulary rows [v0, v0 + v_rows)
-      auto run_d_W = [&](int v0, int v_rows) -> int {
-        UmmaArgs a{};
-        a.M = v_rows; a.N = H; a.K = rows;
-        a.m_tiles = (v_rows + tile_m - 1) / tile_m;
-        a.n_tiles = (H + grad_unit_cols(pl) - 1) / grad_unit_cols(pl);
-        a.group_m = kGradRasterGroup;
-        a.a_mn0 = v0;
-        a.b_k0 = t0;
-        a.row0 = v0;
-        a.d_W = d_W;
-        a.out_ld = (size_t)H;
-        a.accumulate = (panel > 0 || acc_into || pl.compact) ? 1 : 0;
-        a.dyn_rows = n_active; a.dyn_base = t0;
-        a.status = status;
-        return launch_umma<kModeDW>(pl, map_dz_mn, map_hidden_mn, map_dw_out, a, stream);
-      };
-      const bool last_panel = t0 + pl.panel_tokens >= T;
-      if (last_panel && hooks && hooks->after_dw_slab) {
+      if (last_panel && by_slabs) {
         // d_W is final slab by slab, so the caller can start moving it while the rest is computed; a slab
         // is a whole number of waves of units (row tiles in multiples of the worker count), about eight
         const int workers = std::max(1, pl.sms / pl.cta);
@@ -805,17 +834,21 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
         const int slab_rows = slab_tiles * tile_m;
         for (int v0 = 0; v0 < V; v0 += slab_rows) {
           const int v_rows = (V - v0) < slab_rows ? (V - v0) : slab_rows;
-          st = run_d_W(v0, v_rows);
+          st = run_d_W(pn, v0, v_rows);
           if (st != ULORL_OK) return st;
           st = dw_rows_final(v0, v_rows);
           if (st != ULORL_OK) return st;
         }
-        st = run_d_hidden();
+        if (dz_alt) {
+          st = run_d_hidden(held);
+          if (st != ULORL_OK) return st;
+        }
+        st = run_d_hidden(pn);
         if (st != ULORL_OK) return st;
       } else {
-        st = run_d_hidden();
+        st = run_d_hidden(pn);
         if (st != ULORL_OK) return st;
-        st = run_d_W(0, V);
+        st = run_d_W(pn, 0, V);
         if (st != ULORL_OK) return st;
         if (last_panel) {
           st = dw_rows_final(0, V);
@@ -1038,7 +1071,7 @@ int ulorl_kernel_timing_end(float* total_ms, int64_t* launches) {
 namespace {
 struct HostStepLayout {
   size_t hidden, W, targets, old_logp, ref_logp, segver, adv, seq_off, ent_sup;
-  size_t logp, entropy, lse, grad_coef, flags, seq_entropy, loss, stats, d_hidden, d_W, ws, total;
+  size_t logp, entropy, lse, grad_coef, flags, seq_entropy, loss, stats, d_hidden, d_W, ws, dz2, total;
   size_t elem;
 };
 // Two copy streams and a few events, created on the first host-buffer step and kept: the inbound
@@ -1112,7 +1145,11 @@ HostStepLayout host_step_layout(const ulorl_params_t* p) {
   L.stats = take(sizeof(ulorl_stats_t));
   L.d_hidden = take(T * H * L.elem);
   L.d_W = take(V * H * (p->dw_dtype == ULORL_BF16 ? 2 : 4));
-  L.ws = take(make_plan(p).total);
+  const Plan pl = make_plan(p);
+  L.ws = take(pl.total);
+  // a second dz panel when the backward has several panels to reorder at its end (tensor path, dense backward)
+  const bool two_dz = pl.tensor && !pl.compact && p->T > pl.panel_tokens;
+  L.dz2 = two_dz ? take((size_t)pl.panel_tokens * pl.dz_ld * 2) : 0;
   L.total = off;
   return L;
 }
@@ -1256,6 +1293,7 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
       dw_by_slabs = true;
       return (int)ULORL_OK;
     };
+    if (L.dz2) hooks.dz_second_buffer = a + L.dz2;
   }
   st = fwd_impl(params, a + L.hidden, a + L.W, reinterpret_cast<const int32_t*>(a + L.targets),
                 h_old_logp ? reinterpret_cast<const float*>(a + L.old_logp) : nullptr,

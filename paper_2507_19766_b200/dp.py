@@ -149,24 +149,15 @@ def all_reduce_sequence_entropy(table: torch.Tensor) -> torch.Tensor:
     token count) that ulorl_sequence_entropy_partials fills from each rank's pieces.  Integer addition is
     exact, so every rank ends with the sums of the unsplit batch bit for bit; the means are then taken on the
     device by ulorl_sequence_entropy_combine and go to the decision stage as ent_scope = supplied.  This is
-    the one exchange between the forward call and the decision stage that token-range sharding adds."""
+    the one exchange between the forward call and the decision stage that token-range sharding adds.
+
+    The same tables serve the gate of Eq. 10 read as the entropy of the model over one optimiser step: add the
+    tables of the step's micro-batches (integer addition, any order), all-reduce them here, and the batch mean
+    that ulorl_sequence_entropy_combine returns is the token mean entropy of the whole step on every rank; each
+    call of the step then takes it for all of its sequences (ent_scope = supplied), so that micro-batching and
+    sharding do not change which tokens are masked."""
     if table.dtype != torch.int64:
         raise TypeError("the table of per-sequence entropy sums is int64")
     if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
         dist.all_reduce(table)
     return table
-
-
-def step_entropy_gate(call_mean_entropy: Sequence[float], call_tokens: Sequence[int], device=None) -> float:
-    """The gate entropy of Eq. 10 read as the entropy of the model over one optimiser step: the
-    token-weighted mean of the per-call mean entropies (the forward call's mean_entropy statistic) of all
-    micro-batches of this rank and, when a process group is up, of all ranks.  Every call of the step then
-    takes it for each of its sequences (ent_scope = supplied), so that micro-batching and sharding do not
-    change which tokens are masked."""
-    acc = torch.zeros(2, dtype=torch.float64, device=device)
-    for m, n in zip(call_mean_entropy, call_tokens):
-        acc[0] += float(m) * int(n)
-        acc[1] += int(n)
-    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
-        dist.all_reduce(acc)
-    return float(acc[0] / acc[1]) if float(acc[1]) > 0 else 0.0

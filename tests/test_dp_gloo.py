@@ -124,9 +124,9 @@ def _token_range_worker(rank, world, port, result_dir):
         assert np.allclose(gate, full["seq_entropy"][ids].astype(np.float32), rtol=1e-6)
         assert np.array_equal(out["flags"], full["flags"][rows])
         assert np.allclose(out["d_hidden"], full["d_hidden"][rows], rtol=1e-12, atol=1e-15)
-        # the step-wide gate: both ranks obtain the batch mean entropy of the unsplit call
-        step_gate = dp.step_entropy_gate([float(ent32.astype(np.float64).mean())], [rows.size])
-        assert abs(step_gate - full["mean_entropy"]) < 1e-12
+        # the step-wide gate: the same summed table gives both ranks the token mean entropy of the unsplit call
+        step_gate = float(table[:, 0].sum().item()) * 2.0 ** -34 / float(table[:, 1].sum().item())
+        assert abs(step_gate - full["mean_entropy"]) < 1e-9
         if rank == 0:
             assert 0 < full["stats"]["n_masked"] < np.count_nonzero(full["flags"] & O.FLAG_MPT)   # both gate states
             assert np.allclose(d_W.numpy(), full["d_W"], rtol=1e-12, atol=1e-15)
