@@ -252,8 +252,8 @@ class Leg:
         other.__dict__.update(self.__dict__)
         other.gp = dataclasses.replace(self.gp, **kw)
         other.ws = B.alloc_workspace(other.gp, self.ctx.dev)
-        if other.gp.dw_torch_dtype != self.d_W.dtype:
-            other.d_W = torch.empty(self.wl.V, self.wl.H, dtype=other.gp.dw_torch_dtype, device=self.ctx.dev)
+        other.d_hidden = torch.empty_like(self.d_hidden)          # its own gradients: this leg's stay as they are
+        other.d_W = torch.empty(self.wl.V, self.wl.H, dtype=other.gp.dw_torch_dtype, device=self.ctx.dev)
         return other
 
     def step(self, reduce=True):
@@ -383,9 +383,15 @@ def e2e_run(leg: Leg, steps: int, dw_dtype: str) -> dict:
     ctx.fence()
     h2d = sum(t.numel() * t.element_size() for t in hb.values())
     d2h = sum(t.numel() * t.element_size() for t in ho.values())
+    # outside the timed region: the host-buffer step reorders copies and launches, never results -- its
+    # gradients are those of the device-resident step of this leg, bit for bit (a bf16 d_W: its rounding)
+    same_dh = bool(torch.equal(ho["d_hidden"].to(ctx.dev), leg.d_hidden))
+    want_dw = leg.d_W if leg.d_W.dtype == ho["d_W"].dtype else leg.d_W.to(ho["d_W"].dtype)
+    same_dw = bool(torch.equal(ho["d_W"].to(ctx.dev), want_dw))
+    assert same_dh and same_dw, "host-buffer step and device-resident step disagree"
     return {"value": ctx.world * wl.T * steps / dt, "unit": "tokens/s", "ms_per_step": 1e3 * dt / steps,
             "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": steps, "dw_dtype": dw_dtype,
-            "loss": float(ho["loss"][0])}
+            "loss": float(ho["loss"][0]), "gradients_equal_device_step": True}
 
 
 def library_gemm_reference(ctx: Context, seconds: float = 4.0) -> dict:
