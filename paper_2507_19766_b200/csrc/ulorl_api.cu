@@ -12,6 +12,8 @@
 #include <mutex>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "common.cuh"
 #include "elementwise.cuh"
 #include "simt.cuh"
@@ -53,6 +55,16 @@ static int device_sm_count() {
   }
   return sms[dev];
 }
+
+// A named range on the calling host thread for the time its launches are being queued: a timeline tool
+// attached to the process shows which call, pass and panel a kernel belongs to.  Without a tool attached
+// the calls do nothing.
+struct TraceRange {
+  explicit TraceRange(const char* name) { nvtxRangePushA(name); }
+  ~TraceRange() { nvtxRangePop(); }
+  TraceRange(const TraceRange&) = delete;
+  TraceRange& operator=(const TraceRange&) = delete;
+};
 
 struct Plan {
   bool tensor;            // tensor-core path (bf16) or SIMT path
@@ -366,6 +378,7 @@ static int run_decide(const ulorl_params_t* p, const Plan& pl, const float* logp
                       const float* advantages,
                       const int32_t* seq_offsets, const float* entropy_supplied, float* grad_coef, uint8_t* flags,
                       float* seq_entropy, float* loss, void* stats, uint8_t* ws, cudaStream_t stream) {
+  TraceRange trace("ulorl decision stage");
   const int T = p->T, S = p->num_seqs;
   int* status = reinterpret_cast<int*>(ws + pl.off_status);
   float* batch_mean = reinterpret_cast<float*>(ws + pl.off_batch_mean);
@@ -539,6 +552,7 @@ static int fwd_impl(const ulorl_params_t* params, const void* hidden, const void
                     const int32_t* seq_offsets, const float* entropy_supplied, float* logp, float* entropy,
                     float* lse, float* grad_coef, uint8_t* flags, float* seq_entropy, float* loss, void* stats,
                     void* workspace, size_t workspace_bytes, void* cuda_stream, const StepHooks* hooks) {
+  TraceRange trace("ulorl forward");
   int st = validate_params(params);
   if (st != ULORL_OK) return st;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
@@ -658,6 +672,7 @@ static int round_dw_rows(const float* acc, void* d_W, int v0, int v_rows, int H,
 static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void* W, const int32_t* targets,
                     const float* lse, const float* grad_coef, const float* grad_loss, void* d_hidden, void* d_W_out,
                     void* workspace, size_t workspace_bytes, void* cuda_stream, const StepHooks* hooks) {
+  TraceRange trace("ulorl backward");
   int st = validate_params(params);
   if (st != ULORL_OK) return st;
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
@@ -814,6 +829,7 @@ static int bwd_impl(const ulorl_params_t* params, const void* hidden, const void
     Panel held{};
     for (int t0 = 0, panel = 0; t0 < T; t0 += pl.panel_tokens, ++panel) {
       const bool last_panel = panel == n_panels - 1;
+      TraceRange panel_trace(last_panel ? "ulorl backward: last panel" : "ulorl backward: panel");
       Panel pn;
       st = make_panel(t0, panel, (dz_alt && last_panel) ? dz_alt : dz, pn);
       if (st != ULORL_OK) return st;
@@ -1167,6 +1183,7 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
                                const float* h_entropy_supplied, float* h_logp, float* h_entropy, uint8_t* h_flags,
                                float* h_seq_entropy, float* h_loss, void* h_stats, void* h_d_hidden, void* h_d_W,
                                void* d_arena, size_t arena_bytes, void* cuda_stream) {
+  TraceRange trace("ulorl host-buffer step");
   int st = validate_params(params);
   if (st != ULORL_OK) return st;
   if (!d_arena || !h_loss) return ULORL_ERR_INVALID_ARG;

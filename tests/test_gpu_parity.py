@@ -456,16 +456,19 @@ def test_bf16_dw_output_matches_the_oracle_and_the_rounded_f32_result(path, pane
     assert torch.equal(dW, (old.float() + dW32).to(torch.bfloat16))
 
 
-@pytest.mark.parametrize("path,V,panel,dw_dtype", [("tensor", 40000, 512, "f32"), ("tensor", 40000, 512, "bf16"),
-                                                   ("tensor", 2500, 0, "f32"), ("simt", 2500, 256, "f32")])
-def test_backward_reports_dw_slab_by_slab(path, V, panel, dw_dtype):
+@pytest.mark.parametrize("path,V,panel,dw_dtype,compact", [("tensor", 40000, 512, "f32", False),
+                                                           ("tensor", 40000, 512, "bf16", False),
+                                                           ("tensor", 40000, 512, "f32", True),
+                                                           ("tensor", 2500, 0, "f32", False),
+                                                           ("simt", 2500, 256, "f32", False)])
+def test_backward_reports_dw_slab_by_slab(path, V, panel, dw_dtype, compact):
     """ulorl_token_loss_bwd_slabs: the callback sees ascending slabs that cover [0, V) once, the rows it is told
     about are final when the work queued before the callback has run (an event recorded inside the callback
     orders a copy on a second stream), and the results are those of the plain backward bit for bit."""
     wl = synth.WORKLOADS["small"].scaled(T=900, S=4, H=256, V=V, lengths="tiny", planted=0.3,
                                          beta_planted=(100.0, 200.0), mpt_mode="always")
     batch = synth.make_batch(wl, seed=41)
-    gp, _ = both_params(batch, kernel_path=path, bwd_panel_tokens=panel)
+    gp, _ = both_params(batch, kernel_path=path, bwd_panel_tokens=panel, compact_rows=compact)
     import dataclasses
     gp = dataclasses.replace(gp, dw_dtype=dw_dtype)
     out, dH, dW = gpu_fwd_bwd(batch, gp)
