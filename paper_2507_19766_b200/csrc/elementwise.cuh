@@ -79,25 +79,66 @@ __device__ __forceinline__ void checked_range(const int* __restrict__ seq_offset
   }
 }
 
-__global__ void seq_entropy_kernel(int S, int T, const int* __restrict__ seq_offsets, const float* __restrict__ entropy,
-                                   long long* __restrict__ seq_sum, float* __restrict__ seq_entropy, int* __restrict__ status) {
-  const int i = blockIdx.x;
-  int a, b;
-  checked_range(seq_offsets, i, S, T, a, b, status);
-  const long long sum = block_entropy_sum(entropy, a, b);
-  if (threadIdx.x == 0) {
-    seq_sum[i] = sum;
-    if (seq_entropy) seq_entropy[i] = fixed_mean(sum, (long long)(b - a));
+// Step 1: blocks of kSeqChunk consecutive tokens add their entropies into the (zeroed) integer sum of the
+// sequence they belong to.  A block that lies inside one sequence -- nearly all of them, and every one of an
+// ultra-long response -- reduces first and adds once; a block that crosses a boundary adds token by token.
+// Integer addition makes the result independent of how the tokens are grouped.
+constexpr int kSeqChunk = 4096;
+
+__device__ __forceinline__ int sequence_of_token(const int* __restrict__ seq_offsets, int S, int t) {
+  int lo = 0, hi = S;   // largest i with seq_offsets[i] <= t (an empty sequence never owns a token)
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (seq_offsets[mid] <= t) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+__global__ void seq_entropy_sum_kernel(int S, int T, const int* __restrict__ seq_offsets,
+                                       const float* __restrict__ entropy, long long* __restrict__ seq_sum) {
+  const int t0 = blockIdx.x * kSeqChunk;
+  const int t1 = min(T, t0 + kSeqChunk);
+  if (t0 >= t1) return;
+  const int first = sequence_of_token(seq_offsets, S, t0);
+  const int last = sequence_of_token(seq_offsets, S, t1 - 1);
+  if (first == last) {
+    const long long sum = block_entropy_sum(entropy, t0, t1);
+    if (threadIdx.x == 0) atomicAdd(reinterpret_cast<unsigned long long*>(seq_sum + first), (unsigned long long)sum);
+  } else {
+    for (int t = t0 + threadIdx.x; t < t1; t += kSeqThreads) {
+      const int i = sequence_of_token(seq_offsets, S, t);
+      atomicAdd(reinterpret_cast<unsigned long long*>(seq_sum + i), (unsigned long long)entropy_to_fixed(entropy[t]));
+    }
   }
 }
 
-// Token mean of the entropy over the whole call: the (exact) sum of the sequence sums.
-__global__ void batch_entropy_kernel(int S, int T, const long long* __restrict__ seq_sum, float* __restrict__ batch_mean) {
-  if (threadIdx.x == 0 && blockIdx.x == 0) {
-    long long tot = 0;
-    for (int i = 0; i < S; ++i) tot += seq_sum[i];
-    *batch_mean = fixed_mean(tot, (long long)T);
+// Step 2 (one block): the mean of every sequence from its sum and its checked length, and the token mean of
+// the whole call from the (exact) sum of the sequence sums.
+__global__ void seq_entropy_mean_kernel(int S, int T, const int* __restrict__ seq_offsets,
+                                        const long long* __restrict__ seq_sum, float* __restrict__ seq_entropy,
+                                        float* __restrict__ batch_mean, int* __restrict__ status) {
+  __shared__ long long red[kSeqThreads];
+  long long acc = 0;
+  for (int i = threadIdx.x; i < S; i += kSeqThreads) {
+    int a = seq_offsets[i], b = seq_offsets[i + 1];
+    // offsets are device data the host never saw: a bad pair is reported and clamped
+    const bool bad = a < 0 || b < a || b > T || (i == 0 && a != 0) || (i == S - 1 && b != T);
+    if (bad) {
+      if (status) atomicOr(status, kStatusBadOffsets);
+      a = a < 0 ? 0 : (a > T ? T : a);
+      b = b < a ? a : (b > T ? T : b);
+    }
+    const long long sum = seq_sum[i];
+    acc += sum;
+    if (seq_entropy) seq_entropy[i] = fixed_mean(sum, (long long)(b - a));
   }
+  red[threadIdx.x] = acc;
+  __syncthreads();
+  for (int w = kSeqThreads / 2; w > 0; w >>= 1) {
+    if (threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *batch_mean = fixed_mean(red[0], (long long)T);
 }
 
 // The pieces of sequences that one call holds, as rows (sum, count) of a table over ALL sequences of the
@@ -121,7 +162,7 @@ __global__ void seq_entropy_partials_kernel(int S, int T, const int* __restrict_
   }
 }
 
-// Means of the sequences seq_ids[0..n) from a summed table, with the arithmetic of seq_entropy_kernel:
+// Means of the sequences seq_ids[0..n) from a summed table, with the arithmetic of seq_entropy_mean_kernel:
 // a sequence whose pieces were summed here gets the float32 mean the unsplit call would have given it.
 __global__ void seq_entropy_combine_kernel(int n, const int* __restrict__ seq_ids, int total_seqs,
                                            const long long* __restrict__ table, float* __restrict__ seq_entropy,

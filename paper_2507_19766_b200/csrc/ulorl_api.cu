@@ -386,9 +386,10 @@ static int run_decide(const ulorl_params_t* p, const Plan& pl, const float* logp
   DecidePartial* partials = reinterpret_cast<DecidePartial*>(ws + pl.off_decide);
   // the gate needs a float array of per-sequence means even when the caller does not want it back
   float* seq_ent_out = seq_entropy;
-  seq_entropy_kernel<<<S, kSeqThreads, 0, stream>>>(S, T, seq_offsets, entropy, seq_sum, seq_ent_out, status);
+  if (cudaMemsetAsync(seq_sum, 0, sizeof(long long) * (size_t)S, stream) != cudaSuccess) return ULORL_ERR_CUDA;
+  seq_entropy_sum_kernel<<<(T + kSeqChunk - 1) / kSeqChunk, kSeqThreads, 0, stream>>>(S, T, seq_offsets, entropy, seq_sum);
   ULORL_LAUNCH_CHECK();
-  batch_entropy_kernel<<<1, 32, 0, stream>>>(S, T, seq_sum, batch_mean);
+  seq_entropy_mean_kernel<<<1, kSeqThreads, 0, stream>>>(S, T, seq_offsets, seq_sum, seq_ent_out, batch_mean, status);
   ULORL_LAUNCH_CHECK();
   const DecideConsts c = make_decide_consts(p);
   const float* gate = (p->ent_scope == ULORL_ENT_SUPPLIED) ? entropy_supplied : seq_ent_out;
