@@ -213,8 +213,7 @@ __global__ void decide_kernel(int T, int S, DecideConsts c, const float* __restr
                               DecidePartial* __restrict__ partials) {
   __shared__ double sh_loss[kDecideThreads];
   __shared__ double sh_kl[kDecideThreads];
-  __shared__ float sh_abs[kDecideTokens];
-  __shared__ signed char sh_bucket[kDecideTokens];
+  __shared__ double sh_abs_warp[ULORL_N_STALENESS][kDecideThreads / 32];
   __shared__ int sh_cnt[5];
   __shared__ int sh_stale[2][ULORL_N_STALENESS];
   const int tid = threadIdx.x;
@@ -264,7 +263,8 @@ __global__ void decide_kernel(int T, int S, DecideConsts c, const float* __restr
   }
 
   double contrib = 0.0, kl_acc = 0.0;
-  float g4[kDecideVec];
+  float g4[kDecideVec], dabs4[kDecideVec];
+  int bucket4[kDecideVec];
   unsigned f4[kDecideVec];
   int seq = t0 < T ? find_sequence(seq_offsets, S, t0) : 0;
 #pragma unroll
@@ -333,8 +333,8 @@ __global__ void decide_kernel(int T, int S, DecideConsts c, const float* __restr
       atomicAdd(&sh_stale[0][st], 1);
       if (hi || lo) atomicAdd(&sh_stale[1][st], 1);
     }
-    sh_abs[tid * kDecideVec + k] = dabs;
-    sh_bucket[tid * kDecideVec + k] = (signed char)bucket;
+    dabs4[k] = dabs;
+    bucket4[k] = bucket;
   }
   if (whole) {
     if (grad_coef) *reinterpret_cast<float4*>(grad_coef + t0) = make_float4(g4[0], g4[1], g4[2], g4[3]);
@@ -358,10 +358,24 @@ __global__ void decide_kernel(int T, int S, DecideConsts c, const float* __restr
     __syncthreads();
   }
   DecidePartial* out = partials + blockIdx.x;
+  // sum of |log ratio| per staleness bucket, in a fixed order: a thread's tokens in token order, a fixed
+  // butterfly inside each warp, the warps in order; buckets without a token in this block are skipped
+  // (the counts were complete at the barrier above)
+  for (int s = 0; s < ULORL_N_STALENESS; ++s) {
+    if (sh_stale[0][s] == 0 || !sais) continue;
+    double a = 0.0;
+#pragma unroll
+    for (int k = 0; k < kDecideVec; ++k)
+      if (bucket4[k] == s) a += (double)dabs4[k];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
+    if ((tid & 31) == 0) sh_abs_warp[s][tid >> 5] = a;
+  }
+  __syncthreads();
   if (tid < ULORL_N_STALENESS) {
     double a = 0.0;
-    for (int k = 0; k < kDecideTokens; ++k)
-      if (sh_bucket[k] == tid) a += (double)sh_abs[k];
+    if (sh_stale[0][tid] != 0 && sais)
+      for (int w = 0; w < kDecideThreads / 32; ++w) a += sh_abs_warp[tid][w];
     out->stale_abs[tid] = a;
     out->stale_tokens[tid] = sh_stale[0][tid];
     out->stale_clipped[tid] = sh_stale[1][tid];
