@@ -94,8 +94,9 @@ typedef struct {
   int32_t kernel_path;         /* ulorl_kernel_path_t; AUTO = tensor-core path for bf16, SIMT path for f32       */
   int32_t bwd_panel_tokens;    /* bwd: tokens per staging panel; 0 = library default                             */
   int32_t compact_rows;        /* bwd, tensor path: 1 = run the three contractions only on tokens whose          */
-                               /* grad_coef is non-zero (masked, clipped and zero-advantage tokens add nothing   */
-                               /* to either gradient, Eq. 10); results are the same, the workspace grows by two  */
+                               /* grad_coef is non-zero (a masked token, and without a KL term a clipped or      */
+                               /* zero-advantage one, adds nothing to either gradient, Eq. 10); results are the  */
+                               /* same, the workspace grows by two                                               */
                                /* [T, H] copies.  0 = all rows.  Part of the workspace size: pass the same value */
                                /* to ulorl_workspace_bytes and to both calls.                                    */
   int32_t loss_norm;           /* ulorl_loss_norm_t: weight of a token's term in the loss                        */
@@ -109,7 +110,7 @@ typedef struct {
 } ulorl_params_t;
 
 typedef struct {
-  float loss;                  /* -(1/N) sum_t (1 - msk_t) s_t                                                    */
+  float loss;                  /* -(1/N) sum_t (1 - msk_t) (s_t - kl_beta k_t)                                    */
   float mean_entropy;          /* token mean of the per-token entropy over the call                               */
   int32_t n_tokens, n_active, n_mpt, n_masked, n_clip_high, n_clip_low;
   int32_t stale_tokens[ULORL_N_STALENESS];     /* tokens per staleness bucket (last bucket = that or more)        */
@@ -131,7 +132,8 @@ size_t ulorl_workspace_bytes(const ulorl_params_t* params);
  *                          segment (Eq. 8); may be NULL in POIS mode
  *   ref_logp [T] f32       log-prob of the token under the reference policy of Eq. 5's KL term; read only
  *                          when kl_beta > 0, else may be NULL
- *   segment_version [T]    id of that policy (statistics only); may be NULL
+ *   segment_version [T]    id of the policy that generated the token's segment (the map f of Eq. 8; statistics
+ *                          only); may be NULL
  *   advantages             f32, [num_seqs] or [T] (adv_per_token)
  *   seq_offsets [S+1]      int32, non-decreasing, seq_offsets[0] = 0, seq_offsets[S] = T
  *   entropy_supplied [S]   f32 gate values, read only when ent_scope = SUPPLIED
