@@ -1207,7 +1207,7 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
     return (!src || !bytes) ? cudaSuccess : cudaMemcpyAsync(a + off, src, bytes, cudaMemcpyHostToDevice, hs->in);
   };
   if (!ok(h2d(L.targets, h_targets, T * 4)) || !ok(h2d(L.old_logp, h_old_logp, T * 4)) ||
-      !ok(h2d(L.ref_logp, h_ref_logp, T * 4)) ||
+      !ok(h2d(L.ref_logp, h_ref_logp, params->kl_beta > 0.f ? T * 4 : 0)) ||   // unread without the KL term
       !ok(h2d(L.segver, h_segment_version, T * 4)) ||
       !ok(h2d(L.adv, h_advantages, (params->adv_per_token ? T : S) * 4)) ||
       !ok(h2d(L.seq_off, h_seq_offsets, (S + 1) * 4)) || !ok(h2d(L.ent_sup, h_entropy_supplied, S * 4)))
@@ -1315,7 +1315,7 @@ int ulorl_token_loss_step_host(const ulorl_params_t* params, const void* h_hidde
   }
   st = fwd_impl(params, a + L.hidden, a + L.W, reinterpret_cast<const int32_t*>(a + L.targets),
                 h_old_logp ? reinterpret_cast<const float*>(a + L.old_logp) : nullptr,
-                h_ref_logp ? reinterpret_cast<const float*>(a + L.ref_logp) : nullptr,
+                (h_ref_logp && params->kl_beta > 0.f) ? reinterpret_cast<const float*>(a + L.ref_logp) : nullptr,
                 h_segment_version ? reinterpret_cast<const int32_t*>(a + L.segver) : nullptr,
                 reinterpret_cast<const float*>(a + L.adv), reinterpret_cast<const int32_t*>(a + L.seq_off),
                 h_entropy_supplied ? reinterpret_cast<const float*>(a + L.ent_sup) : nullptr,
