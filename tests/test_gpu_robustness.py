@@ -106,3 +106,79 @@ def test_guard_bytes_around_every_buffer_survive_all_passes(path, compact, dw_dt
     assert G.intact()
     assert torch.equal(ho["d_W"], d_W.cpu()) and torch.equal(ho["d_hidden"], d_hidden.cpu())
     assert torch.equal(ho["logp"], out.logp.cpu())
+
+
+def test_decision_stage_with_many_short_and_empty_sequences():
+    """20000 sequences of 0..3 tokens: every thread of the decision kernel steps through several sequence
+    boundaries (and over empty sequences) inside its four tokens, the per-sequence sums take the token-by-token
+    path in every block.  Flags, counts and sequence means against the oracle."""
+    from oracle import ulorl_oracle as O
+    rng = np.random.default_rng(23)
+    S = 20000
+    lens = rng.integers(0, 4, size=S)
+    lens[-1] = max(lens[-1], 1)
+    T = int(lens.sum())
+    offsets = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    logp = (-np.abs(rng.standard_normal(T)) * 0.02).astype(np.float32)
+    logp[rng.random(T) < 0.3] -= np.float32(3.0)
+    ent = (np.abs(rng.standard_normal(T)) * 0.25).astype(np.float32)
+    old = (logp + rng.standard_normal(T).astype(np.float32) * 0.15).astype(np.float32)
+    adv = rng.choice(np.float32([1.0, -1.0, 0.0, 0.7]), size=S).astype(np.float32)
+    version = rng.integers(0, 9, size=T).astype(np.int32)
+    kw = dict(is_mode="sais", mpt_mode="dynamic", entropy_target=0.2, current_version=8)
+    ref = O.decide(logp, O.gate_entropy(ent, offsets, "per_seq", None), old, adv, offsets, version, O.OracleParams(**kw))
+    t = lambda x: torch.from_numpy(x).to(DEV)
+    out = B.token_loss_decide(B.Params(T=T, H=8, V=16, num_seqs=S, dtype="f32", **kw), t(logp), t(ent), t(old),
+                              t(version), t(adv), t(offsets))
+    torch.cuda.synchronize()
+    assert np.array_equal(out.flags.cpu().numpy(), ref["flags"])
+    st = out.stats_host()
+    for k in ("n_tokens", "n_active", "n_mpt", "n_masked", "n_clip_high", "n_clip_low"):
+        assert st[k] == ref["stats"][k], k
+    assert st["device_status"] == 0 and ref["stats"]["n_masked"] > 0
+    seq_mean, batch_mean = O.sequence_mean_entropy(ent, offsets)
+    got = out.seq_entropy.cpu().numpy()[:S]
+    assert np.allclose(got, seq_mean, rtol=1e-6, atol=1e-9) and (got[lens == 0] == 0).all()
+    assert abs(st["mean_entropy"] - batch_mean) <= 1e-6
+    assert np.allclose(out.grad_coef.cpu().numpy(), ref["grad_coef"], rtol=1e-6, atol=0)
+
+
+def test_first_calls_from_two_host_threads_at_once():
+    """Two host threads, each with its own stream, workspace and outputs, make their calls at the same time
+    (ctypes releases the interpreter lock for the duration of a call): the lazily created per-device tables are
+    built under one mutex, and the results are those of the same calls made one after the other."""
+    import threading
+    wl = synth.WORKLOADS["small"].scaled(T=900, S=4, H=256, V=4000, lengths="tiny", planted=0.3,
+                                         beta_planted=(100.0, 200.0), mpt_mode="always")
+    batch = synth.make_batch(wl, seed=18)
+    b = batch.to(DEV)
+    results, errors = {}, []
+
+    def work(name, path):
+        try:
+            gp, _ = both_params(batch, kernel_path=path)
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                ws = B.alloc_workspace(gp, DEV)
+                for _ in range(10):
+                    out = B.token_loss_fwd(gp, b.hidden, b.W, b.targets, b.old_logp, b.segment_version, b.advantages,
+                                           b.seq_offsets, workspace=ws)
+                    dH, dW = B.token_loss_bwd(gp, b.hidden, b.W, b.targets, out.lse, out.grad_coef, workspace=ws)
+                stream.synchronize()
+                assert B.check_status(ws) == B.OK
+            results[name] = (out.logp.clone(), out.loss.clone(), dH.clone(), dW.clone())
+        except BaseException as exc:      # surfaced in the main thread below
+            errors.append(exc)
+
+    torch.cuda.synchronize()
+    threads = [threading.Thread(target=work, args=(f"t{i}", p)) for i, p in enumerate(("tensor", "tensor_1cta", "tensor", "simt"))]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join()
+    assert not errors, errors
+    work("serial_tensor", "tensor")
+    work("serial_1cta", "tensor_1cta")
+    for a, c in (("t0", "serial_tensor"), ("t2", "serial_tensor"), ("t1", "serial_1cta")):
+        for x, y in zip(results[a], results[c]):
+            assert torch.equal(x, y)
